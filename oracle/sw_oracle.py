@@ -1,0 +1,185 @@
+"""ctypes front end of the CPU oracle (``sw_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by ``tests/``, the smoke check and the bench's CPU legs, never by the
+CUDA library or its binding.  It compiles ``sw_oracle.c`` with gcc on first use and marshals numpy
+arrays; all arithmetic is in the C file.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "sw_oracle.c"
+_LIB = _HERE / "libsw_oracle.so"
+_lib = None
+
+F_NO_PREFILL, F_NO_DECODE, F_DECODE_INFEASIBLE, F_CAPPED = 1, 2, 4, 8
+INF = (1 << 63) - 1
+
+
+def build(force: bool = False) -> Path:
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _LIB.with_suffix(f".{os.getpid()}.tmp")
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fopenmp", "-shared", "-fPIC", "-o", str(tmp),
+                               str(_SRC), "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(str(build()))
+        _lib.swo_pool_index.restype = C.c_int64
+        _lib.swo_pool_index.argtypes = [C.c_int64] + [C.c_int] * 7
+        _lib.swo_analytic_cost_ns.restype = C.c_int64
+        _lib.swo_analytic_cost_ns.argtypes = [C.c_int64, C.c_int64]
+        _lib.swo_num_threads.restype = C.c_int
+    return _lib
+
+
+def _p(a, ctype):
+    if a is None:
+        return None
+    return a.ctypes.data_as(C.POINTER(ctype))
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _i64(a):
+    return np.ascontiguousarray(a, dtype=np.int64)
+
+
+def _u16(a):
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.uint16, a.dtype
+    return a
+
+
+def num_threads() -> int:
+    return int(lib().swo_num_threads())
+
+
+def pool_index(page, x, kvh, slot, e, Hkv, S, d) -> int:
+    return int(lib().swo_pool_index(int(page), x, kvh, slot, e, Hkv, S, d))
+
+
+def kv_append(pool, batch, k_new, v_new) -> int:
+    """In-place scatter into ``pool`` (uint16 bits).  Returns the oracle's status code."""
+    sh = batch.shape
+    pool = _u16(pool)
+    pf = _i32(batch.prefill_pages)
+    return int(lib().swo_kv_append(
+        _p(pool, C.c_uint16), C.c_int64(batch.num_pages), sh.num_kv_heads, sh.page_size, sh.head_dim,
+        _p(_u16(k_new), C.c_uint16), _p(_u16(v_new), C.c_uint16),
+        batch.prefix_len, batch.chunk_len, _p(pf, C.c_int32), int(pf.shape[0]),
+        batch.num_decode, _p(_i32(batch.decode_kv_len), C.c_int32),
+        _p(_i32(batch.decode_page_indptr), C.c_int32), _p(_i32(batch.decode_pages), C.c_int32)))
+
+
+def mixed_attention(pool, batch, q, pairs=None, scale: float = 0.0, threads: int = 0):
+    """Attention of a mixed iteration in fp64.
+
+    pairs=None evaluates every (row, head); otherwise ``pairs`` is an int array [m][2] of (row, head).
+    Returns (out [m][d] float64, lse [m] float64, psum [m] float64); with pairs=None the first axis is
+    (C+n)*Hq in row-major order.
+    """
+    sh = batch.shape
+    pool, q = _u16(pool), _u16(q)
+    if pairs is None:
+        m = batch.num_rows * sh.num_q_heads
+        pp = None
+    else:
+        pp = _i32(pairs).reshape(-1, 2)
+        m = pp.shape[0]
+    out = np.zeros((m, sh.head_dim), dtype=np.float64)
+    lse = np.zeros(m, dtype=np.float64)
+    psum = np.zeros(m, dtype=np.float64)
+    pf = _i32(batch.prefill_pages)
+    dl, ip, dp = _i32(batch.decode_kv_len), _i32(batch.decode_page_indptr), _i32(batch.decode_pages)
+    rc = lib().swo_mixed_attention(
+        _p(pool, C.c_uint16), C.c_int64(batch.num_pages), sh.num_q_heads, sh.num_kv_heads, sh.page_size,
+        sh.head_dim, C.c_double(scale), batch.prefix_len, batch.chunk_len, _p(pf, C.c_int32),
+        int(pf.shape[0]), batch.num_decode, _p(dl, C.c_int32), _p(ip, C.c_int32), _p(dp, C.c_int32),
+        _p(q, C.c_uint16), _p(pp, C.c_int32), C.c_int64(m), _p(out, C.c_double), _p(lse, C.c_double),
+        _p(psum, C.c_double), int(threads))
+    if rc != 0:
+        raise RuntimeError(f"oracle swo_mixed_attention failed with status {rc}")
+    return out, lse, psum
+
+
+def dense_causal(q, k, v, Hq, Hkv, d, scale: float = 0.0):
+    q, k, v = _u16(q), _u16(k), _u16(v)
+    T = q.shape[0]
+    out = np.zeros((T, Hq, d), dtype=np.float64)
+    lse = np.zeros((T, Hq), dtype=np.float64)
+    rc = lib().swo_dense_causal(_p(q, C.c_uint16), _p(k, C.c_uint16), _p(v, C.c_uint16), T, Hq, Hkv, d,
+                                C.c_double(scale), _p(out, C.c_double), _p(lse, C.c_double))
+    if rc != 0:
+        raise RuntimeError(f"oracle swo_dense_causal failed with status {rc}")
+    return out, lse
+
+
+class Table:
+    """Raw cost table held as numpy arrays (the oracle keeps no opaque object)."""
+
+    def __init__(self, n_grid, ctx_grid, prefix_grid, chunk_grid, cost_ns, interp: bool = False):
+        self.n_grid, self.ctx_grid = _i32(n_grid), _i64(ctx_grid)
+        self.prefix_grid, self.chunk_grid = _i32(prefix_grid), _i32(chunk_grid)
+        shape = (len(self.n_grid), len(self.ctx_grid), len(self.prefix_grid), len(self.chunk_grid))
+        self.cost = _i64(cost_ns).reshape(shape).copy()
+        self.interp = bool(interp)
+
+    def cummax(self) -> "Table":
+        s = self.cost.shape
+        lib().swo_cummax(_p(self.cost, C.c_int64), s[0], s[1], s[2], s[3])
+        return self
+
+    def _grid_args(self):
+        return (_p(self.n_grid, C.c_int32), len(self.n_grid), _p(self.ctx_grid, C.c_int64), len(self.ctx_grid),
+                _p(self.prefix_grid, C.c_int32), len(self.prefix_grid), _p(self.chunk_grid, C.c_int32),
+                len(self.chunk_grid), _p(self.cost, C.c_int64), int(self.interp))
+
+    def lookup(self, n, ctx, prefix, c) -> int:
+        out = C.c_int64(0)
+        rc = lib().swo_cost_lookup(*self._grid_args(), C.c_int64(n), C.c_int64(ctx), C.c_int64(prefix),
+                                   C.c_int64(c), C.byref(out))
+        if rc != 0:
+            raise IndexError(f"oracle cost lookup out of range (status {rc})")
+        return int(out.value)
+
+    def choose(self, now_ns, deadlines_ns, total_ctx, prefix_len, remaining, c_max=4096, quantum=1,
+               margin_abs_ns=0, margin_ppm=0):
+        """Brute-force Eq. (1).  Returns (chunk, flags, budget_ns)."""
+        dl = _i64(deadlines_ns)
+        chunk, flags, budget = C.c_int32(0), C.c_int32(0), C.c_int64(0)
+        rc = lib().swo_choose_bruteforce(*self._grid_args(), C.c_int64(margin_abs_ns), C.c_int32(margin_ppm),
+                                         C.c_int32(c_max), C.c_int32(quantum), C.c_int64(now_ns),
+                                         _p(dl, C.c_int64), C.c_int32(len(dl)), C.c_int64(total_ctx),
+                                         C.c_int32(prefix_len), C.c_int32(remaining), C.byref(chunk),
+                                         C.byref(flags), C.byref(budget))
+        if rc != 0:
+            raise IndexError(f"oracle chooser failed (status {rc})")
+        return int(chunk.value), int(flags.value), int(budget.value)
+
+
+def analytic_cost_ns(n: int, c: int) -> int:
+    return int(lib().swo_analytic_cost_ns(int(n), int(c)))
+
+
+def analytic_table(n_values, c_max: int) -> Table:
+    """The analytic model tabulated at every integer chunk 0..c_max for the given decode batch sizes."""
+    n_values = sorted(int(x) for x in n_values)
+    chunk_grid = np.arange(0, c_max + 1, dtype=np.int32)
+    cost = np.zeros((len(n_values), 1, 1, len(chunk_grid)), dtype=np.int64)
+    for a, n in enumerate(n_values):
+        for e, c in enumerate(chunk_grid):
+            cost[a, 0, 0, e] = analytic_cost_ns(n, int(c))
+    return Table(n_values, [1 << 40], [1 << 30], chunk_grid, cost)

@@ -1,0 +1,247 @@
+"""Seeded synthetic inputs for the mixed prefill-chunk + decode attention iteration.
+
+This module serves both the CPU oracle's tests and the CUDA path's tests / bench.  It draws shapes,
+lengths, page permutations and tensor values; it contains none of the method's arithmetic (no
+attention, no paging index formula, no chunk choice).  bf16 values travel as uint16 bit patterns so
+that numpy can hold them and both sides see the same bits.
+
+Workload recipes (the paper's workloads are synthetic length distributions; these restate them as
+single-iteration snapshots):
+
+* tiny     8 q heads / 2 KV heads / d=64, 64-page pool, decodes {64,100,180,256}, chunk C=128 at P=256
+* chat     32/8/128, n decodes with contexts uniform in [256, 2048], chunk C at P=512 of a 1024 prompt
+* mixed    32/8/128, 128 decodes with contexts lognormal(median 2048, sigma 1) clipped to [128, 16384]
+* long     32/8/128, 16 decodes with contexts uniform in [32768, 131072], chunk at P=98304
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+
+SEED_BASE = 0x78830000
+
+
+# --------------------------------------------------------------------------------------------
+# bf16 <-> float bit handling (representation only)
+# --------------------------------------------------------------------------------------------
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round float32 to bfloat16 (round-to-nearest-even) and return the uint16 bit patterns."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    u = x.view(np.uint32).astype(np.uint64)
+    rounding = ((u >> 16) & 1) + 0x7FFF
+    out = ((u + rounding) >> 16).astype(np.uint16)
+    nan = np.isnan(x)
+    if nan.any():
+        out = np.where(nan, np.uint16(0x7FC0), out)
+    return out
+
+
+def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    b = np.ascontiguousarray(b, dtype=np.uint16)
+    return (b.astype(np.uint32) << 16).view(np.float32)
+
+
+def bf16_bits_to_f64(b: np.ndarray) -> np.ndarray:
+    return bf16_bits_to_f32(b).astype(np.float64)
+
+
+# --------------------------------------------------------------------------------------------
+# shapes and batches
+# --------------------------------------------------------------------------------------------
+@dataclass(frozen=True)
+class AttnShape:
+    num_q_heads: int
+    num_kv_heads: int
+    head_dim: int
+    page_size: int = 16
+
+    @property
+    def group(self) -> int:
+        return self.num_q_heads // self.num_kv_heads
+
+    @property
+    def page_elems(self) -> int:
+        """bf16 elements of one page (K and V, all KV heads)."""
+        return 2 * self.num_kv_heads * self.page_size * self.head_dim
+
+    @property
+    def token_bytes(self) -> int:
+        return 2 * self.num_kv_heads * self.head_dim * 2
+
+
+TINY = AttnShape(8, 2, 64)
+LLAMA = AttnShape(32, 8, 128)
+
+
+@dataclass
+class MixedBatch:
+    """One mixed iteration: a prefill chunk [P, P+C) of one prompt plus n decode requests.
+
+    ``decode_kv_len[i]`` is the number of keys request i attends, i.e. its context *including* the
+    token whose K/V row is appended in this iteration.  Page lists hold pool page ids.
+    """
+
+    shape: AttnShape
+    num_pages: int
+    prefix_len: int
+    chunk_len: int
+    prefill_pages: np.ndarray  # int32 [ceil((P+C)/page)]
+    decode_kv_len: np.ndarray  # int32 [n]
+    decode_page_indptr: np.ndarray  # int32 [n+1]
+    decode_pages: np.ndarray  # int32 [indptr[n]]
+    name: str = ""
+    meta: dict = field(default_factory=dict)
+
+    @property
+    def num_decode(self) -> int:
+        return int(self.decode_kv_len.shape[0])
+
+    @property
+    def num_rows(self) -> int:
+        return self.chunk_len + self.num_decode
+
+    @property
+    def total_decode_ctx(self) -> int:
+        return int(self.decode_kv_len.astype(np.int64).sum())
+
+
+def _cdiv(a: int, b: int) -> int:
+    return -(-a // b)
+
+
+def make_batch(shape: AttnShape, num_pages: int, decode_lens, prefix_len: int, chunk_len: int,
+               rng: np.random.Generator, name: str = "") -> MixedBatch:
+    """Deal distinct, randomly permuted pool pages to the decodes (in order) and then to the prompt."""
+    decode_lens = np.asarray(decode_lens, dtype=np.int32).reshape(-1)
+    S = shape.page_size
+    per_req = [_cdiv(int(L), S) for L in decode_lens]
+    n_pf = _cdiv(prefix_len + chunk_len, S) if (prefix_len + chunk_len) > 0 else 0
+    need = sum(per_req) + n_pf
+    if need > num_pages:
+        raise ValueError(f"batch needs {need} pages, pool has {num_pages}")
+    if num_pages <= (1 << 22):
+        ids = rng.permutation(num_pages)[:need]
+    else:
+        ids = rng.choice(num_pages, size=need, replace=False)
+    ids = ids.astype(np.int32)
+    indptr = np.zeros(len(per_req) + 1, dtype=np.int32)
+    indptr[1:] = np.cumsum(per_req)
+    return MixedBatch(shape=shape, num_pages=int(num_pages), prefix_len=int(prefix_len),
+                      chunk_len=int(chunk_len), prefill_pages=ids[indptr[-1]:].copy(),
+                      decode_kv_len=decode_lens.copy(), decode_page_indptr=indptr,
+                      decode_pages=ids[:indptr[-1]].copy(), name=name)
+
+
+def normal_bf16_bits(rng: np.random.Generator, *size: int) -> np.ndarray:
+    """N(0,1) drawn in float32 and rounded to bf16 bits."""
+    return f32_to_bf16_bits(rng.standard_normal(size=size, dtype=np.float32))
+
+
+def host_tensors(batch: MixedBatch, rng: np.random.Generator, with_pool: bool = True) -> dict:
+    """Random q / k_new / v_new rows (and the whole pool for small pools), all as bf16 bits.
+
+    Row order everywhere: rows 0..C-1 are the prefill chunk tokens, rows C..C+n-1 the decode tokens.
+    """
+    sh = batch.shape
+    R = batch.num_rows
+    out = {
+        "q": normal_bf16_bits(rng, R, sh.num_q_heads, sh.head_dim),
+        "k_new": normal_bf16_bits(rng, R, sh.num_kv_heads, sh.head_dim),
+        "v_new": normal_bf16_bits(rng, R, sh.num_kv_heads, sh.head_dim),
+    }
+    if with_pool:
+        out["pool"] = normal_bf16_bits(rng, batch.num_pages * sh.page_elems)
+    return out
+
+
+# --------------------------------------------------------------------------------------------
+# the named workloads
+# --------------------------------------------------------------------------------------------
+def rng_for(config_index: int, salt: int = 0) -> np.random.Generator:
+    return np.random.Generator(np.random.PCG64(SEED_BASE + config_index + (salt << 8)))
+
+
+def tiny_batch(rng: np.random.Generator | None = None) -> MixedBatch:
+    rng = rng or rng_for(0)
+    return make_batch(TINY, 64, [64, 100, 180, 256], 256, 128, rng, name="tiny")
+
+
+def chat_batch(n: int = 64, chunk_len: int = 512, prefix_len: int = 512, slack_pages: int = 64,
+               rng: np.random.Generator | None = None) -> MixedBatch:
+    rng = rng or rng_for(1)
+    lens = rng.integers(256, 2048, size=n, endpoint=True)
+    need = int(sum(_cdiv(int(x), 16) for x in lens)) + _cdiv(prefix_len + chunk_len, 16)
+    return make_batch(LLAMA, need + slack_pages, lens, prefix_len, chunk_len, rng, name=f"chat_n{n}_C{chunk_len}")
+
+
+def mixed_lens(n: int, rng: np.random.Generator) -> np.ndarray:
+    raw = np.floor(rng.lognormal(mean=np.log(2048.0), sigma=1.0, size=n))
+    return np.clip(raw, 128, 16384).astype(np.int32)
+
+
+def mixed_batch(chunk_len: int, prefix_len: int, n: int = 128, slack_pages: int = 256,
+                rng: np.random.Generator | None = None) -> MixedBatch:
+    rng = rng or rng_for(2)
+    lens = mixed_lens(n, rng)
+    need = int(sum(_cdiv(int(x), 16) for x in lens)) + _cdiv(prefix_len + chunk_len, 16)
+    return make_batch(LLAMA, need + slack_pages, lens, prefix_len, chunk_len, rng,
+                      name=f"mixed_C{chunk_len}_P{prefix_len}")
+
+
+def long_batch(chunk_len: int, prefix_len: int = 98304, n: int = 16, num_pages: int | None = None,
+               rng: np.random.Generator | None = None) -> MixedBatch:
+    rng = rng or rng_for(3)
+    lens = rng.integers(32768, 131072, size=n, endpoint=True)
+    need = int(sum(_cdiv(int(x), 16) for x in lens)) + _cdiv(prefix_len + chunk_len, 16)
+    if num_pages is None:
+        num_pages = need + 1024
+    return make_batch(LLAMA, int(num_pages), lens, prefix_len, chunk_len, rng,
+                      name=f"long_C{chunk_len}_P{prefix_len}")
+
+
+# --------------------------------------------------------------------------------------------
+# request traces for the bursty controller loop
+# --------------------------------------------------------------------------------------------
+def bursty_trace(num_requests: int = 2000, rate_low: float = 2.0, rate_high: float = 20.0,
+                 mean_dwell_s: float = 10.0, prompt_median: float = 1500.0, prompt_sigma: float = 1.0,
+                 prompt_clip=(32, 32768), mean_output: float = 200.0,
+                 rng: np.random.Generator | None = None) -> dict:
+    """2-state Markov-modulated Poisson arrivals (starting in the low state), lognormal prompt
+    lengths and geometric output lengths.  Times are int64 nanoseconds."""
+    rng = rng or rng_for(4)
+    arrivals = np.empty(num_requests, dtype=np.int64)
+    t = 0.0
+    state_high = False
+    state_end = rng.exponential(mean_dwell_s)
+    i = 0
+    while i < num_requests:
+        rate = rate_high if state_high else rate_low
+        gap = rng.exponential(1.0 / rate)
+        if t + gap >= state_end:
+            # memoryless: jump to the switch point and redraw in the new state
+            t = state_end
+            state_high = not state_high
+            state_end = t + rng.exponential(mean_dwell_s)
+            continue
+        t += gap
+        arrivals[i] = int(round(t * 1e9))
+        i += 1
+    prompts = np.clip(np.floor(rng.lognormal(np.log(prompt_median), prompt_sigma, size=num_requests)),
+                      prompt_clip[0], prompt_clip[1]).astype(np.int32)
+    outputs = rng.geometric(1.0 / mean_output, size=num_requests).astype(np.int32)
+    return {"arrival_ns": arrivals, "prompt_len": prompts, "output_len": outputs}
+
+
+# --------------------------------------------------------------------------------------------
+# device-side fills for pools too large to draw on the host (torch imported lazily)
+# --------------------------------------------------------------------------------------------
+def fill_normal_bf16_(tensor, seed: int, slab_elems: int = 1 << 28) -> None:
+    """Fill a (possibly huge) bf16 torch tensor in place with N(0,1), slab by slab, from one seed."""
+    import torch
+
+    gen = torch.Generator(device=tensor.device)
+    gen.manual_seed(int(seed))
+    flat = tensor.view(-1)
+    for start in range(0, flat.numel(), slab_elems):
+        flat[start:start + slab_elems].normal_(0.0, 1.0, generator=gen)
