@@ -1,0 +1,176 @@
+/*
+ * sloweave — C ABI of the B200 (sm_100a) mixed prefill-chunk + decode attention iteration and of the
+ * SLOWeave chunk controller.
+ *
+ * One serving iteration decodes one token for every active request and optionally processes one
+ * prefill chunk (Sec. 4.1); the controller admits the largest chunk whose predicted iteration cost still
+ * meets the earliest next-token deadline (Sec. 3.1-3.2, Eq. (1), Algorithm 1).  The paper leaves the
+ * attention kernels and the paged KV layout untouched (Sec. 1, Sec. 5.1, Table 1), so the attention itself
+ * is textbook scaled-dot-product attention over a paged bf16 KV cache.
+ *
+ * Conventions
+ *   - Plain C99 types; no exceptions cross the boundary; every call returns an sw_status.
+ *   - "device" pointers are CUDA device memory owned by the caller; the library never frees them and
+ *     allocates no device memory after sw_create (sw_create itself allocates none either: all scratch is
+ *     the caller's workspace).
+ *   - `stream` is a cudaStream_t passed as void*.  Launching calls are asynchronous on that stream.
+ *     One sw_ctx serves one stream at a time (its scratch and counters are shared by its launches).
+ *   - bf16 tensors are dense, row-major, innermost index last.
+ *   - KV pool layout (elements, bf16):  [num_pages][2 (0 = K, 1 = V)][num_kv_heads][page_size][head_dim].
+ *     The pool must hold finite values everywhere a page list can reach (initialise it with zeros): the
+ *     unwritten slots of a partly filled last page are read and multiplied by a zero weight.
+ *   - Row order of q / k_new / v_new / out: rows 0..C-1 are the prefill chunk tokens (chunk token j has
+ *     absolute position P + j), rows C..C+n-1 are the decode tokens of requests 0..n-1.
+ *   - Query head h reads KV head floor(h / (num_q_heads / num_kv_heads)).
+ */
+#ifndef SLOWEAVE_SW_H
+#define SLOWEAVE_SW_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SW_OK = 0,
+    SW_ERR_INVALID_ARG = 1,    /* null pointer, negative size, inconsistent arguments */
+    SW_ERR_OUT_OF_RANGE = 2,   /* page id / length / chunk outside pool, prompt or table grid */
+    SW_ERR_UNSUPPORTED = 3,    /* head_dim, page_size, GQA ratio or device architecture not supported */
+    SW_ERR_WORKSPACE = 4,      /* caller's workspace too small or misaligned */
+    SW_ERR_CUDA = 5,           /* a CUDA runtime / driver call failed; see sw_last_error() */
+    SW_ERR_DEVICE_TIMEOUT = 6, /* a bounded device-side wait gave up */
+    SW_ERR_NOT_MONOTONE = 7    /* cost table not nondecreasing and make_monotone == 0 */
+} sw_status;
+
+typedef struct sw_ctx sw_ctx;               /* opaque; owns tensor-map cache and pointers into the workspace */
+typedef struct sw_cost_table sw_cost_table; /* opaque host object */
+
+/* Attention shape and pool geometry.  Supported: head_dim 64 or 128; page_size 16;
+ * num_q_heads / num_kv_heads in {1, 2, 4, 8}. */
+typedef struct {
+    int32_t num_q_heads, num_kv_heads, head_dim, page_size;
+    int64_t num_pages; /* pages in every pool passed to this context */
+    float sm_scale;    /* softmax scale; <= 0 selects 1/sqrt(head_dim) */
+} sw_layout;
+
+/* One mixed iteration (Sec. 4.1): one prefill chunk of C tokens at cached-prefix offset P of one prompt,
+ * plus the next token of each of n active decodes.  Pointers are DEVICE pointers. */
+typedef struct {
+    int32_t prefix_len;               /* P >= 0 */
+    int32_t chunk_len;                /* C >= 0; 0 = decode-only iteration */
+    const int32_t* prefill_pages;     /* [num_prefill_pages] page ids of the prompt, in order */
+    int32_t num_prefill_pages;        /* >= ceil((P + C) / page_size) */
+    int32_t num_decode;               /* n >= 0; 0 = prefill-only iteration */
+    const int32_t* decode_kv_len;     /* [n] keys attended by request i, INCLUDING the token appended now */
+    const int32_t* decode_page_indptr;/* [n+1] CSR offsets into decode_pages */
+    const int32_t* decode_pages;      /* [indptr[n]] page ids */
+} sw_batch;
+
+/* ---- context -------------------------------------------------------------------------------------- */
+
+/* Bytes of device workspace a context needs for iterations of at most max_chunk chunk tokens and
+ * max_decode decode requests (split-KV partial results, tickets, counters, status words, and staging for
+ * sw_mixed_iteration_host with at most max_pages page-table entries).  Returns 0 on invalid arguments. */
+size_t sw_workspace_bytes(const sw_layout* layout, int32_t max_chunk, int32_t max_decode, int64_t max_pages);
+
+/* Create a context on CUDA device `device`.  `workspace` is device memory of at least
+ * sw_workspace_bytes(...) bytes, 256-byte aligned, owned by the caller and kept alive until sw_destroy.
+ * Its contents are initialised here (synchronously).  Fails with SW_ERR_UNSUPPORTED on a device that is not
+ * compute capability 10.x or on an unsupported shape. */
+sw_status sw_create(const sw_layout* layout, int device, void* workspace, size_t workspace_bytes,
+                    int32_t max_chunk, int32_t max_decode, int64_t max_pages, sw_ctx** out);
+void sw_destroy(sw_ctx* ctx);
+
+/* ---- the hot path ----------------------------------------------------------------------------------- */
+
+/* KV manager step (Table 1): write this iteration's new K/V rows into the pool.  k_new / v_new are device
+ * bf16 [C+n][num_kv_heads][head_dim].  Chunk row j goes to position P+j of the prompt's page list, decode row
+ * i to position decode_kv_len[i]-1 of request i's list.  One kernel launch, asynchronous.  Page ids or
+ * positions outside their list / the pool are skipped and reported by sw_check_status. */
+sw_status sw_kv_append(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const void* k_new, const void* v_new,
+                       void* stream);
+
+/* Executor step (Sec. 4.1; Fig. 1 card 4): attention of the whole mixed iteration in ONE kernel launch —
+ * chunk-prefill tiles on the tensor cores (chunk row j attends keys 0..P+j inclusive), split-KV decode
+ * units and their combine.  q, out: device bf16 [C+n][num_q_heads][head_dim].  lse: device fp32
+ * [C+n][num_q_heads] (natural-log sum-exp of the scaled scores) or NULL.  The K/V of this iteration's rows
+ * must already be in the pool (call sw_kv_append first on the same stream).  Asynchronous. */
+sw_status sw_mixed_attn_run(sw_ctx* ctx, const void* kv_pool, const sw_batch* batch, const void* q, void* out,
+                            float* lse, void* stream);
+
+/* The same iteration from HOST buffers: copies q / k_new / v_new and the page tables to the device (into the
+ * workspace), runs sw_kv_append + sw_mixed_attn_run, copies `out` (and lse if non-NULL) back and waits.
+ * All pointers inside `h_batch` and h_q / h_k_new / h_v_new / h_out / h_lse are HOST pointers (pinned memory
+ * makes the copies asynchronous); kv_pool stays a device pointer. */
+sw_status sw_mixed_iteration_host(sw_ctx* ctx, void* kv_pool, const sw_batch* h_batch, const void* h_q,
+                                  const void* h_k_new, const void* h_v_new, void* h_out, float* h_lse,
+                                  void* stream);
+
+/* Profiler step (Sec. 5.1; Sec. 6.4): time the attention of one iteration over a stack of `layers` pools
+ * (kv_pools: HOST array of `layers` device pool pointers, used round-robin so that successive launches do
+ * not hit the same cache lines).  Runs `warmup` untimed and `reps` timed iterations of `layers` launches
+ * each, timed with CUDA events on `stream`; synchronous.  Returns per-ITERATION nanoseconds: median,
+ * nearest-rank 99th percentile, and (if samples_ns != NULL) all `reps` samples in run order. */
+sw_status sw_cost_probe(sw_ctx* ctx, void* const* kv_pools, int32_t layers, const sw_batch* batch, const void* q,
+                        void* out, int32_t warmup, int32_t reps, int64_t* p50_ns, int64_t* p99_ns,
+                        int64_t* samples_ns, void* stream);
+
+/* Wait for `stream` and read the device status words: *code is 0 or the first device-detected problem as an
+ * sw_status (bad page id / length → SW_ERR_OUT_OF_RANGE, bounded wait expired → SW_ERR_DEVICE_TIMEOUT),
+ * *detail an implementation-defined locator.  The words are cleared.  Returns *code as status. */
+sw_status sw_check_status(sw_ctx* ctx, void* stream, int32_t* code, int32_t* detail);
+
+/* ---- the controller (host only; no CUDA) ---------------------------------------------------------- */
+
+/* Cost table T^(n, ctx, prefix, c) in integer nanoseconds (Sec. 5.1: lookup table indexed by decode batch
+ * size, total cached context and candidate prefill tokens; a prefix-length axis is added).  Grids are
+ * strictly increasing; cost_ns is [nn][nc][np][nk].  make_monotone != 0 applies the cumulative maximum
+ * along the chunk axis (Sec. 5.1) and along the other axes (T is nondecreasing in every argument);
+ * make_monotone == 0 requires the input to be nondecreasing already (else SW_ERR_NOT_MONOTONE).
+ * interp != 0 selects integer-linear interpolation (rounded up) along the chunk axis (Sec. 6.4); otherwise
+ * every coordinate is rounded up to the next grid point. */
+sw_status sw_cost_table_create(const int32_t* n_grid, int32_t nn, const int64_t* ctx_grid, int32_t nc,
+                               const int32_t* prefix_grid, int32_t np, const int32_t* chunk_grid, int32_t nk,
+                               const int64_t* cost_ns, int make_monotone, int interp, sw_cost_table** out);
+void sw_cost_table_destroy(sw_cost_table* table);
+/* Predicted duration; a chunk beyond the last grid point yields INT64_MAX (infeasible); n / ctx / prefix
+ * beyond their grids yield SW_ERR_OUT_OF_RANGE. */
+sw_status sw_cost_table_lookup(const sw_cost_table* table, int64_t n, int64_t ctx, int64_t prefix, int64_t c,
+                               int64_t* cost_ns);
+
+typedef struct {
+    int64_t margin_abs_ns; /* delta = margin_abs_ns + ceil(T^ * margin_ppm / 1e6)  (Sec. 3.3, prediction error) */
+    int32_t margin_ppm;
+    int32_t c_max;         /* C_max, the cap also used when no decode is active (Sec. 3.1) */
+    int32_t chunk_quantum; /* 1 = any integer chunk; q > 1 restricts to multiples of q that are <= L */
+} sw_chooser_params;
+
+#define SW_F_NO_PREFILL 1        /* nothing pending: chunk = 0 */
+#define SW_F_NO_DECODE 2         /* no active decode: chunk = L without consulting the table */
+#define SW_F_DECODE_INFEASIBLE 4 /* even the decode-only iteration misses the earliest deadline */
+#define SW_F_CAPPED 8            /* c_max < remaining */
+
+typedef struct {
+    int32_t chunk;        /* chosen c* */
+    int32_t flags;        /* SW_F_* */
+    int64_t budget_ns;    /* B = max(0, min_i d_i - now) */
+    int64_t predicted_ns; /* T^ + delta at the chosen chunk (INT64_MAX never; 0 when no table query was made) */
+    int32_t queries;      /* cost-model queries made by the bisection */
+} sw_choice;
+
+/* Algorithm 1: P empty -> 0; L = min(C_max, remaining); A empty -> L; B = min_i(d_i) - now; upper-mid
+ * bisection over [0, L] on T^ + delta <= B.  deadlines_ns are absolute next-token deadlines d_i = l_i + D_i
+ * (HOST array, n_active entries).  remaining_prefill = 0 means no pending prefill. */
+sw_status sw_choose_chunk(const sw_cost_table* table, const sw_chooser_params* params, int64_t now_ns,
+                          const int64_t* deadlines_ns, int32_t n_active, int64_t total_ctx, int32_t prefix_len,
+                          int32_t remaining_prefill, sw_choice* out);
+
+/* Thread-local text describing the last non-OK status returned on this thread ("" if none). */
+const char* sw_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLOWEAVE_SW_H */

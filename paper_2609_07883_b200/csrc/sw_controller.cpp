@@ -1,0 +1,212 @@
+// Host controller: monotone cost table and the deadline-aware chunk chooser (Algorithm 1).
+// Pure host code; integer-nanosecond arithmetic so that ties are exact.
+#include <algorithm>
+#include <cstdint>
+#include <cstdio>
+#include <limits>
+#include <new>
+#include <vector>
+
+#include "sw.h"
+#include "sw_error.h"
+
+struct sw_cost_table {
+    std::vector<int32_t> n_grid;
+    std::vector<int64_t> ctx_grid;
+    std::vector<int32_t> prefix_grid;
+    std::vector<int32_t> chunk_grid;
+    std::vector<int64_t> cost;  // [nn][nc][np][nk]
+    bool interp = false;
+
+    size_t at(size_t a, size_t b, size_t c, size_t e) const {
+        return ((a * ctx_grid.size() + b) * prefix_grid.size() + c) * chunk_grid.size() + e;
+    }
+};
+
+namespace {
+
+constexpr int64_t kInf = std::numeric_limits<int64_t>::max();
+
+template <class T>
+bool strictly_increasing(const std::vector<T>& g) {
+    for (size_t i = 1; i < g.size(); ++i)
+        if (!(g[i - 1] < g[i])) return false;
+    return true;
+}
+
+// Running maximum along one axis of the 4-D table; returns true if anything changed.
+bool running_max_axis(sw_cost_table& t, int axis) {
+    const size_t dims[4] = {t.n_grid.size(), t.ctx_grid.size(), t.prefix_grid.size(), t.chunk_grid.size()};
+    bool changed = false;
+    size_t idx[4];
+    for (idx[0] = 0; idx[0] < dims[0]; ++idx[0])
+        for (idx[1] = 0; idx[1] < dims[1]; ++idx[1])
+            for (idx[2] = 0; idx[2] < dims[2]; ++idx[2])
+                for (idx[3] = 0; idx[3] < dims[3]; ++idx[3]) {
+                    if (idx[axis] == 0) continue;
+                    size_t prev[4] = {idx[0], idx[1], idx[2], idx[3]};
+                    prev[axis] -= 1;
+                    int64_t& cur = t.cost[t.at(idx[0], idx[1], idx[2], idx[3])];
+                    const int64_t before = t.cost[t.at(prev[0], prev[1], prev[2], prev[3])];
+                    if (cur < before) {
+                        cur = before;
+                        changed = true;
+                    }
+                }
+    return changed;
+}
+
+// delta(T) = margin_abs + ceil(T * ppm / 1e6); infinity stays infinity.
+int64_t add_margin(int64_t t, const sw_chooser_params& p) {
+    if (t == kInf) return kInf;
+    const __int128 rel = ((__int128)t * p.margin_ppm + 999999) / 1000000;
+    const __int128 sum = (__int128)t + p.margin_abs_ns + rel;
+    return sum >= (__int128)kInf ? kInf : (int64_t)sum;
+}
+
+// index of the first grid point >= x, or grid.size() when x lies beyond the grid
+template <class T>
+size_t round_up_index(const std::vector<T>& grid, int64_t x) {
+    return (size_t)(std::lower_bound(grid.begin(), grid.end(), x,
+                                     [](const T& g, int64_t v) { return (int64_t)g < v; }) -
+                    grid.begin());
+}
+
+sw_status lookup(const sw_cost_table& t, int64_t n, int64_t ctx, int64_t prefix, int64_t c, int64_t* out) {
+    const size_t a = round_up_index(t.n_grid, n);
+    const size_t b = round_up_index(t.ctx_grid, ctx);
+    const size_t p = round_up_index(t.prefix_grid, prefix);
+    if (a == t.n_grid.size() || b == t.ctx_grid.size() || p == t.prefix_grid.size())
+        return sw_fail(SW_ERR_OUT_OF_RANGE, "cost lookup: n=%lld ctx=%lld prefix=%lld beyond the table grid",
+                       (long long)n, (long long)ctx, (long long)prefix);
+    const size_t e = round_up_index(t.chunk_grid, c);
+    if (e == t.chunk_grid.size()) {
+        *out = kInf;
+        return SW_OK;
+    }
+    const int64_t hi = t.cost[t.at(a, b, p, e)];
+    if (!t.interp || e == 0 || (int64_t)t.chunk_grid[e] == c) {
+        *out = hi;
+        return SW_OK;
+    }
+    const int64_t lo = t.cost[t.at(a, b, p, e - 1)];
+    const int64_t c_lo = t.chunk_grid[e - 1], c_hi = t.chunk_grid[e];
+    const __int128 rise = (__int128)(hi - lo) * (c - c_lo);
+    const __int128 span = c_hi - c_lo;
+    *out = lo + (int64_t)((rise + span - 1) / span);  // hi >= lo: table is monotone
+    return SW_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+sw_status sw_cost_table_create(const int32_t* n_grid, int32_t nn, const int64_t* ctx_grid, int32_t nc,
+                               const int32_t* prefix_grid, int32_t np, const int32_t* chunk_grid, int32_t nk,
+                               const int64_t* cost_ns, int make_monotone, int interp, sw_cost_table** out) {
+    if (!n_grid || !ctx_grid || !prefix_grid || !chunk_grid || !cost_ns || !out)
+        return sw_fail(SW_ERR_INVALID_ARG, "sw_cost_table_create: null argument");
+    if (nn < 1 || nc < 1 || np < 1 || nk < 1)
+        return sw_fail(SW_ERR_INVALID_ARG, "sw_cost_table_create: every axis needs at least one grid point");
+    sw_cost_table* t = new (std::nothrow) sw_cost_table();
+    if (!t) return sw_fail(SW_ERR_INVALID_ARG, "sw_cost_table_create: out of host memory");
+    t->n_grid.assign(n_grid, n_grid + nn);
+    t->ctx_grid.assign(ctx_grid, ctx_grid + nc);
+    t->prefix_grid.assign(prefix_grid, prefix_grid + np);
+    t->chunk_grid.assign(chunk_grid, chunk_grid + nk);
+    t->cost.assign(cost_ns, cost_ns + (size_t)nn * nc * np * nk);
+    t->interp = interp != 0;
+    bool ok = strictly_increasing(t->n_grid) && strictly_increasing(t->ctx_grid) &&
+              strictly_increasing(t->prefix_grid) && strictly_increasing(t->chunk_grid) && t->chunk_grid[0] >= 0 &&
+              t->n_grid[0] >= 0 && t->ctx_grid[0] >= 0 && t->prefix_grid[0] >= 0;
+    for (int64_t v : t->cost) ok = ok && v >= 0 && v < (int64_t(1) << 62);
+    if (!ok) {
+        delete t;
+        return sw_fail(SW_ERR_INVALID_ARG,
+                       "sw_cost_table_create: grids must be non-negative and strictly increasing, costs in [0, 2^62)");
+    }
+    // chunk axis first (the profiler's rule), then prefix, ctx, n; repeat until stable so that the result is
+    // nondecreasing along every axis at once.
+    bool changed = false;
+    for (int round = 0; round < 8; ++round) {
+        bool any = false;
+        for (int axis = 3; axis >= 0; --axis) any = running_max_axis(*t, axis) || any;
+        changed = changed || any;
+        if (!any) break;
+    }
+    if (changed && !make_monotone) {
+        delete t;
+        return sw_fail(SW_ERR_NOT_MONOTONE, "sw_cost_table_create: table is not nondecreasing and make_monotone == 0");
+    }
+    *out = t;
+    return SW_OK;
+}
+
+void sw_cost_table_destroy(sw_cost_table* table) { delete table; }
+
+sw_status sw_cost_table_lookup(const sw_cost_table* table, int64_t n, int64_t ctx, int64_t prefix, int64_t c,
+                               int64_t* cost_ns) {
+    if (!table || !cost_ns) return sw_fail(SW_ERR_INVALID_ARG, "sw_cost_table_lookup: null argument");
+    if (n < 0 || ctx < 0 || prefix < 0 || c < 0)
+        return sw_fail(SW_ERR_INVALID_ARG, "sw_cost_table_lookup: negative coordinate");
+    return lookup(*table, n, ctx, prefix, c, cost_ns);
+}
+
+sw_status sw_choose_chunk(const sw_cost_table* table, const sw_chooser_params* params, int64_t now_ns,
+                          const int64_t* deadlines_ns, int32_t n_active, int64_t total_ctx, int32_t prefix_len,
+                          int32_t remaining_prefill, sw_choice* out) {
+    if (!params || !out) return sw_fail(SW_ERR_INVALID_ARG, "sw_choose_chunk: null argument");
+    if (n_active < 0 || remaining_prefill < 0 || prefix_len < 0 || total_ctx < 0 || params->c_max < 0 ||
+        params->margin_ppm < 0 || params->margin_abs_ns < 0 || (n_active > 0 && !deadlines_ns))
+        return sw_fail(SW_ERR_INVALID_ARG, "sw_choose_chunk: negative size or missing deadlines");
+    const int32_t q = params->chunk_quantum > 1 ? params->chunk_quantum : 1;
+    *out = sw_choice{0, 0, 0, 0, 0};
+    // P empty -> 0
+    if (remaining_prefill == 0) {
+        out->flags = SW_F_NO_PREFILL;
+        return SW_OK;
+    }
+    // L = min(C_max, remaining(r))
+    const int32_t L = std::min(params->c_max, remaining_prefill);
+    if (params->c_max < remaining_prefill) out->flags |= SW_F_CAPPED;
+    // A empty -> L
+    if (n_active == 0) {
+        out->chunk = L - L % q;
+        out->flags |= SW_F_NO_DECODE;
+        return SW_OK;
+    }
+    if (!table) return sw_fail(SW_ERR_INVALID_ARG, "sw_choose_chunk: a cost table is required when decodes are active");
+    // B = min_i (l_i + D - s), clamped at zero (Sec. 3.1)
+    const int64_t earliest = *std::min_element(deadlines_ns, deadlines_ns + n_active);
+    const int64_t B = earliest > now_ns ? earliest - now_ns : 0;
+    out->budget_ns = B;
+
+    int64_t t_raw = 0;
+    sw_status st = lookup(*table, n_active, total_ctx, prefix_len, 0, &t_raw);
+    if (st != SW_OK) return st;
+    const int64_t decode_only = add_margin(t_raw, *params);
+    if (decode_only > B) out->flags |= SW_F_DECODE_INFEASIBLE;
+    out->predicted_ns = decode_only;
+
+    // upper-mid bisection over k in [0, L/q], candidate chunk c = k*q
+    int32_t lo = 0, hi = L / q;
+    int64_t predicted_at_lo = decode_only;
+    while (lo < hi) {
+        const int32_t mid = lo + (hi - lo + 1) / 2;
+        st = lookup(*table, n_active, total_ctx, prefix_len, (int64_t)mid * q, &t_raw);
+        if (st != SW_OK) return st;
+        out->queries += 1;
+        const int64_t t = add_margin(t_raw, *params);
+        if (t <= B) {
+            lo = mid;
+            predicted_at_lo = t;
+        } else {
+            hi = mid - 1;
+        }
+    }
+    out->chunk = lo * q;
+    out->predicted_ns = predicted_at_lo;
+    return SW_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,75 @@
+// Internal definitions shared by the library's host code and kernels (not part of the ABI).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sw.h"
+
+namespace sw {
+
+constexpr int kPageSize = 16;           // tokens per page
+constexpr int kMaxDecode = 2048;        // decode requests per iteration (prefix-sum array lives in shared memory)
+constexpr int kThreads = 384;           // 12 warps per CTA, one CTA per SM
+constexpr int kWarps = kThreads / 32;
+constexpr int kTargetItems = 4096;      // split-KV units aimed at per launch (bounds the partial-result scratch)
+constexpr int kMinSplitTokens = 256;    // never split a decode context finer than this
+constexpr int kMaxGroup = 8;            // query heads per KV head
+
+// Control words at the start of the workspace.
+enum CtrlWord { kCtrWork = 0, kCtrDone = 1, kCtrStatus = 2, kCtrDetail = 3, kCtrWords = 64 };
+
+// Device-detected problem locators written to kCtrDetail (high byte = site, low 24 bits = index).
+enum DetailSite { kSiteAppendPage = 1, kSiteAppendLen = 2, kSiteAttnLen = 3, kSiteAttnPage = 4, kSiteWait = 5,
+                  kSiteScratch = 6, kSiteTmem = 7 };
+
+struct MixedParams {
+    // shape
+    int Hq, Hkv, group;
+    int64_t num_pages;
+    float sm_scale;       // softmax scale
+    float sm_scale_log2;  // sm_scale * log2(e)
+    // batch
+    int P, C, n;
+    const int32_t* prefill_pages;
+    int num_prefill_pages;
+    const int32_t* decode_kv_len;
+    const int32_t* decode_page_indptr;
+    const int32_t* decode_pages;
+    const __nv_bfloat16* q;
+    __nv_bfloat16* out;
+    float* lse;
+    // scratch
+    int32_t* ctrl;
+    int32_t* tickets;   // [max_decode * Hkv]
+    float* part_ml;     // [max_items][2 * kMaxGroup]  (m then l per query head of the group)
+    float* part_o;      // [max_items][group * D]
+    int max_items;      // partial-result slots available
+    int target_items;   // split-KV units aimed at (<= max_items - n*Hkv)
+    int prefill_rows_on_decode_path;  // bring-up switch: run every chunk row as a one-token unit
+};
+
+struct AppendParams {
+    int Hkv, D;
+    int64_t num_pages;
+    int P, C, n;
+    const int32_t* prefill_pages;
+    int num_prefill_pages;
+    const int32_t* decode_kv_len;
+    const int32_t* decode_page_indptr;
+    const int32_t* decode_pages;
+    const __nv_bfloat16* k_new;
+    const __nv_bfloat16* v_new;
+    __nv_bfloat16* pool;
+    int32_t* ctrl;
+};
+
+// launchers (sw_kernels.cu)
+cudaError_t launch_kv_append(const AppendParams& p, cudaStream_t stream);
+cudaError_t launch_mixed_attn(int head_dim, const CUtensorMap& kv_map, const MixedParams& p, int num_sms,
+                              cudaStream_t stream);
+cudaError_t configure_kernels(int head_dim);
+size_t mixed_attn_smem_bytes(int head_dim);
+
+}  // namespace sw

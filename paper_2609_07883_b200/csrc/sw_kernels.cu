@@ -1,0 +1,547 @@
+// sm_100a kernels of the mixed prefill-chunk + decode attention iteration.
+//
+//   sw_kv_append_kernel     scatter of this iteration's new K/V rows into their pages (Table 1, KV manager)
+//   sw_mixed_attn_kernel    ONE persistent launch per iteration (Sec. 4.1): every CTA plans the split-KV units
+//                           from the context lengths, warps pull units from a shared counter, stream K/V pages
+//                           with TMA into a per-warp shared-memory ring, keep an online softmax in registers and
+//                           the last-arriving warp of a request merges its partial results.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "sw_internal.h"
+#include "sw_ptx.cuh"
+
+namespace sw {
+using namespace swptx;
+
+// ---------------------------------------------------------------------------------------------------------------
+// device status: first problem wins
+// ---------------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void report(int32_t* ctrl, int code, int site, int index) {
+    if (atomicCAS(&ctrl[kCtrStatus], 0, code) == 0) ctrl[kCtrDetail] = (site << 24) | (index & 0xFFFFFF);
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// KV append
+// ---------------------------------------------------------------------------------------------------------------
+// One thread per (row, 16-byte piece of the row's Hkv*D elements); it copies that piece of K and of V.
+__global__ void sw_kv_append_kernel(const AppendParams p) {
+    const int pieces_per_row = p.Hkv * p.D / 8;
+    const int64_t total = (int64_t)(p.C + p.n) * pieces_per_row;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+        const int row = (int)(idx / pieces_per_row);
+        const int piece = (int)(idx % pieces_per_row);
+        int64_t pos;
+        const int32_t* pages;
+        int npages;
+        if (row < p.C) {
+            pos = (int64_t)p.P + row;
+            pages = p.prefill_pages;
+            npages = p.num_prefill_pages;
+        } else {
+            const int i = row - p.C;
+            const int len = p.decode_kv_len[i];
+            if (len < 1) {
+                report(p.ctrl, SW_ERR_OUT_OF_RANGE, kSiteAppendLen, i);
+                continue;
+            }
+            pos = (int64_t)len - 1;
+            const int beg = p.decode_page_indptr[i];
+            pages = p.decode_pages + beg;
+            npages = p.decode_page_indptr[i + 1] - beg;
+        }
+        const int64_t pi = pos / kPageSize;
+        const int slot = (int)(pos % kPageSize);
+        if (pi >= npages) {
+            report(p.ctrl, SW_ERR_OUT_OF_RANGE, kSiteAppendLen, row);
+            continue;
+        }
+        const int64_t page = pages[pi];
+        if (page < 0 || page >= p.num_pages) {
+            report(p.ctrl, SW_ERR_OUT_OF_RANGE, kSiteAppendPage, row);
+            continue;
+        }
+        const int e0 = piece * 8;          // element offset inside the row's [Hkv][D]
+        const int kvh = e0 / p.D;
+        const int e = e0 % p.D;
+        const int64_t src = (int64_t)row * p.Hkv * p.D + e0;
+        const int64_t dst_k = ((((int64_t)page * 2 + 0) * p.Hkv + kvh) * kPageSize + slot) * p.D + e;
+        const int64_t dst_v = ((((int64_t)page * 2 + 1) * p.Hkv + kvh) * kPageSize + slot) * p.D + e;
+        *reinterpret_cast<uint4*>(p.pool + dst_k) = *reinterpret_cast<const uint4*>(p.k_new + src);
+        *reinterpret_cast<uint4*>(p.pool + dst_v) = *reinterpret_cast<const uint4*>(p.v_new + src);
+    }
+}
+
+cudaError_t launch_kv_append(const AppendParams& p, cudaStream_t stream) {
+    const int64_t total = (int64_t)(p.C + p.n) * (p.Hkv * p.D / 8);
+    if (total == 0) return cudaSuccess;
+    const int threads = 256;
+    int64_t blocks = (total + threads - 1) / threads;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    sw_kv_append_kernel<<<(unsigned)blocks, threads, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// mixed attention: shared-memory plan
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int kStages = 2;  // K/V page buffers in flight per warp
+
+template <int D>
+struct Geo {
+    static constexpr int kHalves = D / 64;                    // 128-byte swizzled column blocks per row
+    static constexpr int kBlockBytes = kPageSize * 128;       // one [16 tokens][64 elems] swizzled block
+    static constexpr int kStageBytes = 2 * kHalves * kBlockBytes;  // K then V of one (page, kv head)
+    static constexpr int kRingBytes = kWarps * kStages * kStageBytes;
+    static constexpr int kBarOffset = kRingBytes;                              // kWarps*kStages mbarriers
+    static constexpr int kPlanOffset = kBarOffset + kWarps * kStages * 8;      // int32 unit_prefix[kMaxDecode+1]
+    static constexpr int kMiscOffset = kPlanOffset + (kMaxDecode + 1) * 4;     // scan scratch etc.
+    static constexpr int kSmemBytes = kMiscOffset + 256;
+};
+
+struct Plan {
+    int split_tokens;   // tokens per split-KV unit (multiple of the page size)
+    int decode_units;   // sum over requests of ceil(len / split_tokens)
+    int prefill_items;  // chunk-row units on the decode path (bring-up)
+    int total_items;
+};
+
+// Block-wide exclusive scan of one value per thread (kThreads threads).  scratch: kWarps+1 ints.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* scratch, int* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) scratch[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        int w = lane < kWarps ? scratch[lane] : 0;
+        int winc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, winc, o);
+            if (lane >= o) winc += t;
+        }
+        if (lane < kWarps) scratch[lane] = winc - w;
+        if (lane == kWarps - 1) scratch[kWarps] = winc;
+    }
+    __syncthreads();
+    const int r = scratch[warp] + inc - v;
+    *total = scratch[kWarps];
+    __syncthreads();
+    return r;
+}
+
+// Every CTA derives the same plan from the context lengths: no host planning, no extra launch.
+__device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix, int* scratch) {
+    Plan plan;
+    const int per_thread = (p.n + kThreads - 1) / kThreads;
+    const int beg = min(p.n, (int)threadIdx.x * per_thread);
+    const int end = min(p.n, beg + per_thread);
+    // total context in pages (fits an int: n <= 2048 requests of < 2^27 pages)
+    int pages_local = 0;
+    for (int i = beg; i < end; ++i) {
+        const int len = p.decode_kv_len[i];
+        pages_local += len > 0 ? (len + kPageSize - 1) / kPageSize : 0;
+    }
+    int total_pages = 0;
+    block_exclusive_scan(pages_local, scratch, &total_pages);
+    const int per_head_target = max(1, p.target_items / p.Hkv);
+    int split_pages = (total_pages + per_head_target - 1) / per_head_target;
+    split_pages = max(split_pages, kMinSplitTokens / kPageSize);
+    plan.split_tokens = split_pages * kPageSize;
+    int units_local = 0;
+    for (int i = beg; i < end; ++i) {
+        const int len = p.decode_kv_len[i];
+        units_local += len > 0 ? (len + plan.split_tokens - 1) / plan.split_tokens : 0;
+    }
+    int total_units = 0;
+    int run = block_exclusive_scan(units_local, scratch, &total_units);
+    for (int i = beg; i < end; ++i) {
+        unit_prefix[i] = run;
+        const int len = p.decode_kv_len[i];
+        run += len > 0 ? (len + plan.split_tokens - 1) / plan.split_tokens : 0;
+    }
+    if (threadIdx.x == 0) unit_prefix[p.n] = total_units;
+    __syncthreads();
+    plan.decode_units = total_units;
+    plan.prefill_items = p.prefill_rows_on_decode_path ? p.C * p.Hkv : 0;
+    plan.total_items = plan.prefill_items + total_units * p.Hkv;
+    return plan;
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// one split-KV unit on one warp
+// ---------------------------------------------------------------------------------------------------------------
+struct Unit {
+    int q_row;          // row of q / out
+    int kvh;            // KV head
+    int len;            // keys attended by this row in total
+    int t_begin, t_end; // this unit's key range
+    int nsplit;         // units of this (row, kv head); 1 = write the result directly
+    int split;          // index among them
+    int ticket;         // ticket slot (decode request * Hkv + kvh)
+    int slot;           // partial-result slot
+    const int32_t* pages;
+};
+
+template <int D>
+struct WarpRing {
+    uint32_t buf;   // shared address of this warp's first stage
+    uint32_t bar;   // shared address of this warp's first mbarrier
+    uint32_t it;    // pages consumed so far (stage = it % kStages, parity = (it / kStages) & 1)
+};
+
+template <int D>
+__device__ __forceinline__ void issue_page(const CUtensorMap* kv_map, const WarpRing<D>& ring, uint32_t issue_it, int page,
+                                           int kvh, int Hkv) {
+    const uint32_t stage = issue_it % kStages;
+    const uint32_t dst = ring.buf + stage * Geo<D>::kStageBytes;
+    const uint32_t bar = ring.bar + stage * 8;
+    mbar_arrive_expect_tx(bar, Geo<D>::kStageBytes);
+#pragma unroll
+    for (int x = 0; x < 2; ++x)
+#pragma unroll
+        for (int h = 0; h < Geo<D>::kHalves; ++h)
+            tma_load_4d(dst + (x * Geo<D>::kHalves + h) * Geo<D>::kBlockBytes, kv_map, bar, h * 64, 0, x * Hkv + kvh, page);
+}
+
+// Runs one unit; returns false if a bounded wait expired.
+template <int D>
+__device__ bool run_unit(const CUtensorMap* kv_map, const MixedParams& p, const Unit& u, WarpRing<D>& ring) {
+    constexpr int KS = D / 16;  // k-slices of QK^T; also pairs of 8-wide output column tiles of PV
+    const int lane = threadIdx.x & 31;
+    const int qrow_in_group = lane >> 2;  // accumulator row held in c0/c1
+    const int g = p.group;
+
+    // A fragments of Q: rows 0..g-1 are the query heads sharing this KV head, rows >= g are zero
+    uint32_t qa[KS][2];
+    {
+        const __nv_bfloat16* qbase = p.q + ((int64_t)u.q_row * p.Hq + (int64_t)u.kvh * g) * D;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            uint32_t v0 = 0, v1 = 0;
+            if (qrow_in_group < g) {
+                const uint32_t* src = reinterpret_cast<const uint32_t*>(qbase + qrow_in_group * D + ks * 16 + (lane & 3) * 2);
+                v0 = src[0];
+                v1 = src[4];  // +8 elements
+            }
+            qa[ks][0] = v0;
+            qa[ks][1] = v1;
+        }
+    }
+
+    float o[2 * KS][2];
+#pragma unroll
+    for (int i = 0; i < 2 * KS; ++i) o[i][0] = o[i][1] = 0.f;
+    float m_run = -INFINITY, l_run = 0.f;
+
+    const int pg0 = u.t_begin / kPageSize;
+    const int pg1 = (u.t_end + kPageSize - 1) / kPageSize;
+    const int npg = pg1 - pg0;
+
+    // per-lane shared-memory offsets of the ldmatrix rows (128-byte swizzle: 16-byte chunk ^= row % 8)
+    const int k_tok = ((lane >> 4) << 3) + (lane & 7);
+    const int k_sel = (lane >> 3) & 1;
+    const int v_tok = (((lane >> 3) & 1) << 3) + (lane & 7);
+    const int v_sel = lane >> 4;
+    const int swz = lane & 7;
+
+    int ids = 0;
+    int issued = 0;
+    auto issue_next = [&]() {
+        if ((issued & 31) == 0) {
+            const int pi = pg0 + issued + lane;
+            ids = pi < pg1 ? u.pages[pi] : 0;
+        }
+        const int page = __shfl_sync(0xffffffffu, ids, issued & 31);
+        if (page < 0 || (int64_t)page >= p.num_pages) {
+            if (lane == 0) report(p.ctrl, SW_ERR_OUT_OF_RANGE, kSiteAttnPage, u.q_row);
+        }
+        if (lane == 0) issue_page<D>(kv_map, ring, ring.it + issued, page, u.kvh, p.Hkv);
+        ++issued;
+    };
+    for (int k = 0; k < kStages && k < npg; ++k) issue_next();
+
+    for (int k = 0; k < npg; ++k) {
+        const uint32_t stage = ring.it % kStages;
+        const uint32_t parity = (ring.it / kStages) & 1;
+        const uint32_t sK = ring.buf + stage * Geo<D>::kStageBytes;
+        const uint32_t sV = sK + Geo<D>::kHalves * Geo<D>::kBlockBytes;
+        if (!mbar_wait(ring.bar + stage * 8, parity)) {
+            report(p.ctrl, SW_ERR_DEVICE_TIMEOUT, kSiteWait, u.q_row);
+            return false;
+        }
+        const int t0 = (pg0 + k) * kPageSize;
+
+        // S = Q K^T for 16 keys
+        float s[2][4];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            const int chunk = 2 * ks + k_sel;
+            const uint32_t addr = sK + (chunk >> 3) * Geo<D>::kBlockBytes + k_tok * 128 + (((chunk & 7) ^ swz) << 4);
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4(addr, b0, b1, b2, b3);
+            mma_bf16_16816(s[0], qa[ks][0], 0u, qa[ks][1], 0u, b0, b1);
+            mma_bf16_16816(s[1], qa[ks][0], 0u, qa[ks][1], 0u, b2, b3);
+        }
+        // mask keys outside [t_begin, t_end)
+        const int valid_hi = u.t_end - t0;   // keys with index >= valid_hi are masked
+        const int valid_lo = u.t_begin - t0; // keys with index <  valid_lo are masked (always <= 0 here)
+        float mx = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int key = nt * 8 + (lane & 3) * 2 + j;
+                const float v = (key < valid_hi && key >= valid_lo) ? s[nt][j] : -INFINITY;
+                s[nt][j] = v;
+                mx = fmaxf(mx, v);
+            }
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float m_new = fmaxf(m_run, mx);
+        const float corr = fast_exp2((m_run - m_new) * p.sm_scale_log2);
+        const float mb = m_new * p.sm_scale_log2;
+        float pr[2][2];
+        float psum = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                pr[nt][j] = fast_exp2(fmaf(s[nt][j], p.sm_scale_log2, -mb));
+                psum += pr[nt][j];
+            }
+        l_run = l_run * corr + psum;
+        m_run = m_new;
+#pragma unroll
+        for (int i = 0; i < 2 * KS; ++i) {
+            o[i][0] *= corr;
+            o[i][1] *= corr;
+        }
+        const uint32_t pa0 = pack_bf16x2(pr[0][0], pr[0][1]);
+        const uint32_t pa2 = pack_bf16x2(pr[1][0], pr[1][1]);
+
+        // the unwritten slots of a partly filled last page hold whatever the pool held: zero those V rows so that
+        // 0 * garbage cannot produce NaN
+        if (valid_hi < kPageSize) {
+            __syncwarp();
+            const int dead_rows = kPageSize - valid_hi;
+            for (int c = lane; c < dead_rows * (D / 8); c += 32) {
+                const int row = valid_hi + c / (D / 8);
+                const int chunk = c % (D / 8);
+                const uint32_t addr = sV + (chunk >> 3) * Geo<D>::kBlockBytes + row * 128 + (((chunk & 7) ^ (row & 7)) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
+            }
+            __syncwarp();
+        }
+
+        // O += P V
+#pragma unroll
+        for (int dn = 0; dn < KS; ++dn) {
+            const int chunk = 2 * dn + v_sel;
+            const uint32_t addr = sV + (chunk >> 3) * Geo<D>::kBlockBytes + v_tok * 128 + (((chunk & 7) ^ swz) << 4);
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4_trans(addr, b0, b1, b2, b3);
+            float acc0[4] = {o[2 * dn][0], o[2 * dn][1], 0.f, 0.f};
+            float acc1[4] = {o[2 * dn + 1][0], o[2 * dn + 1][1], 0.f, 0.f};
+            mma_bf16_16816(acc0, pa0, 0u, pa2, 0u, b0, b1);
+            mma_bf16_16816(acc1, pa0, 0u, pa2, 0u, b2, b3);
+            o[2 * dn][0] = acc0[0];
+            o[2 * dn][1] = acc0[1];
+            o[2 * dn + 1][0] = acc1[0];
+            o[2 * dn + 1][1] = acc1[1];
+        }
+        ring.it += 1;
+        __syncwarp();  // every lane is done reading this stage before it is refilled
+        if (valid_hi < kPageSize) fence_proxy_async_smem();
+        if (issued < npg) issue_next();
+    }
+
+    // finish: row sums across the quad
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    const bool row_ok = qrow_in_group < g;
+    const int head = u.kvh * g + qrow_in_group;
+    if (u.nsplit == 1) {
+        if (row_ok) {
+            const float inv = 1.f / l_run;
+            __nv_bfloat16* dst = p.out + ((int64_t)u.q_row * p.Hq + head) * D + (lane & 3) * 2;
+#pragma unroll
+            for (int i = 0; i < 2 * KS; ++i)
+                *reinterpret_cast<uint32_t*>(dst + i * 8) = pack_bf16x2(o[i][0] * inv, o[i][1] * inv);
+            if (p.lse && (lane & 3) == 0) p.lse[(int64_t)u.q_row * p.Hq + head] = m_run * p.sm_scale + __logf(l_run);
+        }
+        return true;
+    }
+
+    // partial result -> scratch, then ticket; the last arriver merges
+    if (row_ok) {
+        float* po = p.part_o + ((int64_t)u.slot * g + qrow_in_group) * D + (lane & 3) * 2;
+#pragma unroll
+        for (int i = 0; i < 2 * KS; ++i) *reinterpret_cast<float2*>(po + i * 8) = make_float2(o[i][0], o[i][1]);
+        if ((lane & 3) == 0) {
+            p.part_ml[(int64_t)u.slot * (2 * kMaxGroup) + qrow_in_group] = m_run;
+            p.part_ml[(int64_t)u.slot * (2 * kMaxGroup) + kMaxGroup + qrow_in_group] = l_run;
+        }
+    }
+    __threadfence();
+    __syncwarp();
+    int prev = 0;
+    if (lane == 0) prev = atomicAdd(&p.tickets[u.ticket], 1);
+    prev = __shfl_sync(0xffffffffu, prev, 0);
+    if (prev != u.nsplit - 1) return true;
+
+    // last arriver: merge all splits of this (request, kv head); slots of its splits are Hkv apart
+    __threadfence();
+    if (lane == 0) p.tickets[u.ticket] = 0;  // ready for the next launch
+    const int slot0 = u.slot - u.split * p.Hkv;
+    for (int r = 0; r < g; ++r) {
+        float m_all = -INFINITY;
+        for (int sidx = 0; sidx < u.nsplit; ++sidx)
+            m_all = fmaxf(m_all, __ldcg(&p.part_ml[(int64_t)(slot0 + sidx * p.Hkv) * (2 * kMaxGroup) + r]));
+        float l_all = 0.f;
+        float acc[D / 32];
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) acc[c] = 0.f;
+        for (int sidx = 0; sidx < u.nsplit; ++sidx) {
+            const int64_t sl = slot0 + sidx * p.Hkv;
+            const float ms = __ldcg(&p.part_ml[sl * (2 * kMaxGroup) + r]);
+            const float ls = __ldcg(&p.part_ml[sl * (2 * kMaxGroup) + kMaxGroup + r]);
+            const float w = fast_exp2((ms - m_all) * p.sm_scale_log2);
+            l_all += ls * w;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) acc[c] += w * __ldcg(&p.part_o[(sl * g + r) * D + c * 32 + lane]);
+        }
+        const float inv = 1.f / l_all;
+        const int hd = u.kvh * g + r;
+        __nv_bfloat16* dst = p.out + ((int64_t)u.q_row * p.Hq + hd) * D;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) dst[c * 32 + lane] = __float2bfloat16(acc[c] * inv);
+        if (p.lse && lane == 0) p.lse[(int64_t)u.q_row * p.Hq + hd] = m_all * p.sm_scale + __logf(l_all);
+    }
+    return true;
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// the persistent kernel
+// ---------------------------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid_constant__ CUtensorMap kv_map,
+                                                                    const MixedParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    int* unit_prefix = reinterpret_cast<int*>(smem + Geo<D>::kPlanOffset);
+    int* scratch = reinterpret_cast<int*>(smem + Geo<D>::kMiscOffset);
+
+    if (threadIdx.x == 0) {
+        tma_prefetch_desc(&kv_map);
+        for (int i = 0; i < kWarps * kStages; ++i) mbar_init(base + Geo<D>::kBarOffset + i * 8, 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+
+    const Plan plan = make_plan(p, unit_prefix, scratch);
+    if (plan.total_items > p.max_items + plan.prefill_items) {
+        if (threadIdx.x == 0) report(p.ctrl, SW_ERR_WORKSPACE, kSiteScratch, plan.total_items);
+    } else {
+        WarpRing<D> ring;
+        ring.buf = base + warp * kStages * Geo<D>::kStageBytes;
+        ring.bar = base + Geo<D>::kBarOffset + warp * kStages * 8;
+        ring.it = 0;
+        while (true) {
+            int item = 0;
+            if (lane == 0) item = atomicAdd(&p.ctrl[kCtrWork], 1);
+            item = __shfl_sync(0xffffffffu, item, 0);
+            if (item >= plan.total_items) break;
+            Unit u;
+            bool ok = true;
+            if (item < plan.prefill_items) {
+                const int j = item / p.Hkv;
+                u.q_row = j;
+                u.kvh = item % p.Hkv;
+                u.len = p.P + j + 1;
+                u.t_begin = 0;
+                u.t_end = u.len;
+                u.nsplit = 1;
+                u.split = 0;
+                u.ticket = 0;
+                u.slot = 0;
+                u.pages = p.prefill_pages;
+                ok = (u.len + kPageSize - 1) / kPageSize <= p.num_prefill_pages;
+            } else {
+                const int di = item - plan.prefill_items;
+                const int unit = di / p.Hkv;
+                u.kvh = di % p.Hkv;
+                int lo = 0, hi = p.n;  // largest i with unit_prefix[i] <= unit
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (unit_prefix[mid] <= unit) lo = mid; else hi = mid;
+                }
+                const int i = lo;
+                u.q_row = p.C + i;
+                u.len = p.decode_kv_len[i];
+                u.split = unit - unit_prefix[i];
+                u.nsplit = unit_prefix[i + 1] - unit_prefix[i];
+                u.t_begin = u.split * plan.split_tokens;
+                u.t_end = min(u.len, u.t_begin + plan.split_tokens);
+                u.ticket = i * p.Hkv + u.kvh;
+                u.slot = di;
+                const int beg = p.decode_page_indptr[i];
+                u.pages = p.decode_pages + beg;
+                ok = (u.len + kPageSize - 1) / kPageSize <= p.decode_page_indptr[i + 1] - beg;
+            }
+            if (!ok) {
+                if (lane == 0) report(p.ctrl, SW_ERR_OUT_OF_RANGE, kSiteAttnLen, u.q_row);
+                continue;
+            }
+            if (!run_unit<D>(&kv_map, p, u, ring)) break;
+        }
+    }
+
+    // the last CTA to finish re-arms the work counter for the next launch
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const int done = atomicAdd(&p.ctrl[kCtrDone], 1);
+        if (done == (int)gridDim.x - 1) {
+            p.ctrl[kCtrWork] = 0;
+            p.ctrl[kCtrDone] = 0;
+            __threadfence();
+        }
+    }
+}
+
+size_t mixed_attn_smem_bytes(int head_dim) {
+    return (head_dim == 64 ? Geo<64>::kSmemBytes : Geo<128>::kSmemBytes) + 1024;
+}
+
+cudaError_t configure_kernels(int head_dim) {
+    if (head_dim == 64)
+        return cudaFuncSetAttribute(sw_mixed_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)mixed_attn_smem_bytes(64));
+    return cudaFuncSetAttribute(sw_mixed_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)mixed_attn_smem_bytes(128));
+}
+
+cudaError_t launch_mixed_attn(int head_dim, const CUtensorMap& kv_map, const MixedParams& p, int num_sms,
+                              cudaStream_t stream) {
+    const size_t smem = mixed_attn_smem_bytes(head_dim);
+    if (head_dim == 64)
+        sw_mixed_attn_kernel<64><<<num_sms, kThreads, smem, stream>>>(kv_map, p);
+    else
+        sw_mixed_attn_kernel<128><<<num_sms, kThreads, smem, stream>>>(kv_map, p);
+    return cudaGetLastError();
+}
+
+}  // namespace sw

@@ -1,0 +1,136 @@
+"""sw_choose_chunk (Algorithm 1, bisection) against the oracle's exhaustive Eq. (1) scan: bit-exact."""
+from pathlib import Path
+
+import numpy as np
+import pytest
+
+MS = 1_000_000
+GOLDEN = Path(__file__).resolve().parent / "golden"
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2609_07883_b200 import build
+
+    build.build()
+    from paper_2609_07883_b200 import binding
+
+    return binding
+
+
+def both_tables(B, oracle, n_grid, ctx_grid, prefix_grid, chunk_grid, cost, interp=False, monotone=True):
+    lib_t = B.CostTable(n_grid, ctx_grid, prefix_grid, chunk_grid, cost, make_monotone=monotone, interp=interp)
+    ora_t = oracle.Table(n_grid, ctx_grid, prefix_grid, chunk_grid, cost, interp=interp)
+    if monotone:
+        ora_t.cummax()
+    return lib_t, ora_t
+
+
+def random_table(rng, monotone_input):
+    nn, nc, np_ = (int(rng.integers(1, 4)) for _ in range(3))
+    nk = int(rng.integers(2, 10))
+    n_grid = np.cumsum(rng.integers(1, 50, size=nn))
+    ctx_grid = np.cumsum(rng.integers(1, 10**6, size=nc)).astype(np.int64)
+    prefix_grid = np.cumsum(rng.integers(0, 5000, size=np_)) + np.arange(np_)
+    chunk_grid = np.cumsum(rng.integers(1, 300, size=nk))
+    if rng.integers(0, 2):
+        chunk_grid[0] = 0
+    cost = rng.integers(50_000, 30 * MS, size=(nn, nc, np_, nk)).astype(np.int64)
+    if monotone_input:
+        for ax in range(4):
+            cost = np.maximum.accumulate(cost, axis=ax)
+    return n_grid, ctx_grid, prefix_grid, chunk_grid, cost
+
+
+def test_tables_agree_with_oracle_lookup(B, oracle):
+    rng = np.random.default_rng(100)
+    for trial in range(30):
+        grids = random_table(rng, monotone_input=False)
+        interp = bool(trial % 2)
+        lt, ot = both_tables(B, oracle, *grids, interp=interp)
+        n_grid, ctx_grid, prefix_grid, chunk_grid, _ = grids
+        for _ in range(200):
+            n = int(rng.integers(0, n_grid[-1] + 1))
+            ctx = int(rng.integers(0, ctx_grid[-1] + 1))
+            pre = int(rng.integers(0, prefix_grid[-1] + 1))
+            c = int(rng.integers(0, chunk_grid[-1] + 40))
+            assert lt.lookup(n, ctx, pre, c) == ot.lookup(n, ctx, pre, c)
+        with pytest.raises(B.SwError) as e:
+            lt.lookup(int(n_grid[-1]) + 1, 0, 0, 0)
+        assert e.value.status == B.SW_ERR_OUT_OF_RANGE
+
+
+@pytest.mark.parametrize("interp", [False, True])
+def test_bisection_equals_exhaustive_scan_on_random_monotone_tables(B, oracle, interp):
+    rng = np.random.default_rng(200 + int(interp))
+    for trial in range(60):
+        grids = random_table(rng, monotone_input=bool(trial % 2))
+        lt, ot = both_tables(B, oracle, *grids, interp=interp)
+        n_grid, ctx_grid, prefix_grid, chunk_grid, _ = grids
+        values = sorted(set(int(v) for v in ot.cost.reshape(-1)))
+        budgets = [0, 1] + [v + d for v in values[:: max(1, len(values) // 12)] for d in (-1, 0, 1)] + [10**12]
+        for budget in budgets:
+            n = int(rng.integers(1, n_grid[-1] + 1))
+            ctx = int(rng.integers(0, ctx_grid[-1] + 1))
+            pre = int(rng.integers(0, prefix_grid[-1] + 1))
+            remaining = int(rng.integers(1, chunk_grid[-1] + 60))
+            c_max = int(rng.choice([64, 512, 4096]))
+            quantum = int(rng.choice([1, 1, 16]))
+            ppm = int(rng.choice([0, 50_000]))
+            mabs = int(rng.choice([0, 12_345]))
+            now = int(rng.integers(0, 10**9))
+            dl = now + budget + rng.integers(0, 5 * MS, size=n)
+            dl[rng.integers(0, n)] = now + budget
+            got = B.sw_choose_chunk(lt, now, dl, ctx, pre, remaining, c_max=c_max, chunk_quantum=quantum,
+                                    margin_abs_ns=mabs, margin_ppm=ppm)
+            want = ot.choose(now, dl, ctx, pre, remaining, c_max=c_max, quantum=quantum, margin_abs_ns=mabs,
+                             margin_ppm=ppm)
+            assert (got.chunk, got.flags, got.budget_ns) == want, (trial, budget)
+            L = min(c_max, remaining) // quantum
+            assert got.queries <= max(1, int(np.ceil(np.log2(L + 1)))) if L > 0 else got.queries == 0
+
+
+def test_branch_cases_and_flags(B, oracle):
+    table = oracle.analytic_table([4], 4096)
+    lt = B.CostTable(table.n_grid, table.ctx_grid, table.prefix_grid, table.chunk_grid, table.cost)
+    now = 10 * MS
+    dl = np.array([now + 25 * MS] * 4)
+    r = B.sw_choose_chunk(lt, now, dl, 4, 0, 0)
+    assert (r.chunk, r.flags, r.queries) == (0, B.SW_F_NO_PREFILL, 0)
+    r = B.sw_choose_chunk(None, now, [], 10**15, 10**9, 9000, c_max=4096)      # no table needed without decodes
+    assert (r.chunk, r.flags, r.queries) == (4096, B.SW_F_NO_DECODE | B.SW_F_CAPPED, 0)
+    r = B.sw_choose_chunk(lt, now, dl - 40 * MS, 4, 0, 512)
+    assert r.chunk == 0 and r.budget_ns == 0 and r.flags & B.SW_F_DECODE_INFEASIBLE
+    r = B.sw_choose_chunk(lt, now, dl + 10**12, 4, 0, 3000)
+    assert r.chunk == 3000 and r.flags == 0
+    t = oracle.analytic_cost_ns(4, 100)
+    assert B.sw_choose_chunk(lt, 0, [t] * 4, 4, 0, 4096).chunk == 100
+    assert B.sw_choose_chunk(lt, 0, [t] * 4, 4, 0, 4096).predicted_ns == t
+    assert B.sw_choose_chunk(lt, 0, [t - 1] * 4, 4, 0, 4096).chunk == 99
+    with pytest.raises(B.SwError) as e:
+        B.sw_choose_chunk(lt, 0, [t] * 5, 5, 0, 4096)     # n = 5 beyond the table's n grid
+    assert e.value.status == B.SW_ERR_OUT_OF_RANGE
+
+
+def test_golden_closed_form_chunks(B, oracle):
+    for line in (GOLDEN / "analytic_model_chunks.txt").read_text().splitlines():
+        if not line.strip() or line.startswith("#"):
+            continue
+        n, budget, L, want_chunk, want_inf = (int(x) for x in line.split())
+        table = oracle.analytic_table([n], 4096)
+        lt = B.CostTable(table.n_grid, table.ctx_grid, table.prefix_grid, table.chunk_grid, table.cost)
+        r = B.sw_choose_chunk(lt, 7, [7 + budget] * n, n * 500, 0, L, c_max=4096)
+        assert r.chunk == want_chunk
+        assert bool(r.flags & B.SW_F_DECODE_INFEASIBLE) == bool(want_inf)
+
+
+def test_raw_non_monotone_table_breaks_bisection_and_cummax_restores_it(B, oracle):
+    rows = [[int(x) for x in l.split()] for l in (GOLDEN / "cummax_worked_example.txt").read_text().splitlines()
+            if l.strip() and not l.startswith("#")]
+    grid, raw = rows[0], rows[1]
+    with pytest.raises(B.SwError) as e:
+        B.CostTable([1], [10], [0], grid, raw, make_monotone=False)
+    assert e.value.status == B.SW_ERR_NOT_MONOTONE
+    lt = B.CostTable([1], [10], [0], grid, raw, make_monotone=True)
+    for budget, _want_raw, want_mono in rows[3:]:
+        assert B.sw_choose_chunk(lt, 0, [budget], 10, 0, 112, c_max=112).chunk == want_mono
