@@ -135,7 +135,7 @@ class Context:
         self.handle = handle
 
     def close(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and _lib is not None:
             _lib.sw_destroy(self.handle)
             self.handle = None
 
@@ -237,7 +237,7 @@ class CostTable:
         return int(out.value)
 
     def close(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and _lib is not None:
             _lib.sw_cost_table_destroy(self.handle)
             self.handle = None
 

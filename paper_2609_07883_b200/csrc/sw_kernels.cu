@@ -253,6 +253,7 @@ __device__ bool run_unit(const CUtensorMap* kv_map, const MixedParams& p, const 
 
     int ids = 0;
     int issued = 0;
+    const uint32_t it0 = ring.it;  // ring position of this unit's first page
     auto issue_next = [&]() {
         if ((issued & 31) == 0) {
             const int pi = pg0 + issued + lane;
@@ -262,7 +263,7 @@ __device__ bool run_unit(const CUtensorMap* kv_map, const MixedParams& p, const 
         if (page < 0 || (int64_t)page >= p.num_pages) {
             if (lane == 0) report(p.ctrl, SW_ERR_OUT_OF_RANGE, kSiteAttnPage, u.q_row);
         }
-        if (lane == 0) issue_page<D>(kv_map, ring, ring.it + issued, page, u.kvh, p.Hkv);
+        if (lane == 0) issue_page<D>(kv_map, ring, it0 + issued, page, u.kvh, p.Hkv);
         ++issued;
     };
     for (int k = 0; k < kStages && k < npg; ++k) issue_next();

@@ -1,0 +1,225 @@
+"""GPU parity: the CUDA path, called through the C-ABI, against the fp64 oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+
+from paper_2609_07883_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import torch
+
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_07883_b200 import build
+
+    build.build()
+    from tests import gpu_util
+
+    return gpu_util
+
+
+def run_and_compare(gpu, oracle, batch, tensors, pairs=None, what=""):
+    r = gpu.Runner(batch, tensors)
+    r.append()
+    r.attend()
+    out, lse = r.results()
+    assert r.status() == (0, 0), f"{what}: device status {r.status()}"
+    # oracle on its own copy of the pool, appended by the oracle
+    pool = tensors["pool"].copy()
+    assert oracle.kv_append(pool, batch, tensors["k_new"], tensors["v_new"]) == 0
+    assert np.array_equal(gpu.torch_to_bits(r.pool), pool), f"{what}: pool differs after append"
+    sh = batch.shape
+    if pairs is None:
+        ref, ref_lse, _ = oracle.mixed_attention(pool, batch, tensors["q"])
+        g = out.reshape(-1, sh.head_dim)
+        gl = lse.reshape(-1)
+    else:
+        pairs = np.asarray(pairs, dtype=np.int32)
+        ref, ref_lse, _ = oracle.mixed_attention(pool, batch, tensors["q"], pairs=pairs)
+        g = out[pairs[:, 0], pairs[:, 1]]
+        gl = lse[pairs[:, 0], pairs[:, 1]]
+    return gpu.compare(g, gl, ref, ref_lse, what)
+
+
+def test_tiny_workload_full(gpu, oracle):
+    rng = W.rng_for(0)
+    batch = W.tiny_batch(rng)
+    t = W.host_tensors(batch, rng)
+    run_and_compare(gpu, oracle, batch, t, what="tiny")
+
+
+@pytest.mark.parametrize("shape", [W.TINY, W.AttnShape(8, 2, 128), W.AttnShape(4, 4, 64), W.AttnShape(8, 1, 128),
+                                   W.AttnShape(4, 2, 128)])
+def test_ragged_small_cases(gpu, oracle, shape):
+    rng = np.random.default_rng(31)
+    lens = [1, 15, 16, 17, 31, 255, 256, 257, 700]
+    batch = W.make_batch(shape, 160, lens, 37, 91, rng)
+    t = W.host_tensors(batch, rng)
+    run_and_compare(gpu, oracle, batch, t, what=f"ragged {shape}")
+
+
+def test_decode_only_and_prefill_only(gpu, oracle):
+    rng = np.random.default_rng(32)
+    b1 = W.make_batch(W.TINY, 64, [5, 300, 77], 0, 0, rng)
+    run_and_compare(gpu, oracle, b1, W.host_tensors(b1, rng), what="decode-only")
+    b2 = W.make_batch(W.TINY, 64, [], 130, 70, rng)
+    run_and_compare(gpu, oracle, b2, W.host_tensors(b2, rng), what="prefill-only")
+    b3 = W.make_batch(W.TINY, 64, [], 0, 33, rng)
+    run_and_compare(gpu, oracle, b3, W.host_tensors(b3, rng), what="prefill at P=0")
+
+
+def test_long_decode_is_split_and_merged(gpu, oracle):
+    """Contexts far above the minimum split length exercise the split-KV units and the last-arriver merge."""
+    rng = np.random.default_rng(33)
+    lens = [9000, 4097, 12345, 300]
+    need = sum(-(-x // 16) for x in lens)
+    batch = W.make_batch(W.AttnShape(8, 2, 128), need + 8, lens, 0, 0, rng)
+    t = W.host_tensors(batch, rng)
+    run_and_compare(gpu, oracle, batch, t, what="split decode")
+    # twice in a row on one context: tickets and counters must re-arm themselves
+    r = gpu.Runner(batch, t)
+    r.append()
+    r.attend()
+    first, _ = r.results()
+    r.out.zero_()
+    r.attend()
+    second, _ = r.results()
+    assert np.array_equal(first, second)
+
+
+def test_length_one_rows_return_v0_bit_exactly(gpu, oracle):
+    rng = np.random.default_rng(34)
+    batch = W.make_batch(W.TINY, 32, [1, 1, 40], 0, 3, rng)
+    t = W.host_tensors(batch, rng)
+    r = gpu.Runner(batch, t)
+    r.append()
+    r.attend()
+    out_bits = gpu.torch_to_bits(r.out)
+    g = batch.shape.group
+    for h in range(batch.shape.num_q_heads):
+        assert np.array_equal(out_bits[0, h], t["v_new"][0, h // g])      # chunk row 0 at P = 0
+        assert np.array_equal(out_bits[3, h], t["v_new"][3, h // g])      # decode with one key
+        assert np.array_equal(out_bits[4, h], t["v_new"][4, h // g])
+
+
+def test_nan_in_unwritten_slots_of_the_last_page_does_not_leak(gpu, oracle):
+    rng = np.random.default_rng(35)
+    batch = W.make_batch(W.AttnShape(8, 2, 128), 64, [5, 33, 250], 20, 45, rng)
+    t = W.host_tensors(batch, rng)
+    t["pool"][:] = 0x7FC0  # every slot NaN until written
+    # fill the already-cached positions (prefix and earlier decode tokens) with finite values
+    pool = t["pool"]
+    pv = pool.reshape(batch.num_pages, 2, 2, 16, 128)
+    S = 16
+    for pos in range(batch.prefix_len):
+        pv[batch.prefill_pages[pos // S], :, :, pos % S, :] = W.normal_bf16_bits(rng, 2, 2, 128)
+    for i, L in enumerate(batch.decode_kv_len):
+        pages = batch.decode_pages[batch.decode_page_indptr[i]:]
+        for pos in range(int(L) - 1):
+            pv[pages[pos // S], :, :, pos % S, :] = W.normal_bf16_bits(rng, 2, 2, 128)
+    run_and_compare(gpu, oracle, batch, t, what="NaN tail")
+
+
+def test_page_permutation_invariance(gpu, oracle):
+    rng = np.random.default_rng(36)
+    shape = W.AttnShape(8, 2, 128)
+    outs = []
+    for seed in (1, 2):
+        batch = W.make_batch(shape, 96, [100, 333], 50, 60, np.random.default_rng(seed))
+        trng = np.random.default_rng(99)
+        t = W.host_tensors(batch, trng, with_pool=False)
+        t["pool"] = np.zeros(batch.num_pages * shape.page_elems, np.uint16)
+        # write the cached history through the oracle-independent append of the CUDA path itself: first an
+        # iteration that appends the history, then the iteration under test
+        hist = W.MixedBatch(shape, batch.num_pages, 0, 50, batch.prefill_pages[:4].copy(), np.zeros(0, np.int32),
+                            np.zeros(1, np.int32), np.zeros(0, np.int32))
+        hk = W.normal_bf16_bits(np.random.default_rng(7), 50, 2, 128)
+        hv = W.normal_bf16_bits(np.random.default_rng(8), 50, 2, 128)
+        assert oracle.kv_append(t["pool"], hist, hk, hv) == 0
+        for i, L in enumerate(batch.decode_kv_len):
+            one = W.MixedBatch(shape, batch.num_pages, 0, int(L) - 1,
+                               batch.decode_pages[batch.decode_page_indptr[i]:batch.decode_page_indptr[i + 1]].copy(),
+                               np.zeros(0, np.int32), np.zeros(1, np.int32), np.zeros(0, np.int32))
+            dk = W.normal_bf16_bits(np.random.default_rng(10 + i), int(L) - 1, 2, 128)
+            dv = W.normal_bf16_bits(np.random.default_rng(20 + i), int(L) - 1, 2, 128)
+            assert oracle.kv_append(t["pool"], one, dk, dv) == 0
+        r = gpu.Runner(batch, t)
+        r.append()
+        r.attend()
+        outs.append(gpu.torch_to_bits(r.out).copy())
+        run_and_compare(gpu, oracle, batch, t, what=f"perm {seed}")
+    assert np.array_equal(outs[0], outs[1])
+
+
+def test_bad_page_ids_are_reported_not_faulted(gpu, oracle):
+    rng = np.random.default_rng(37)
+    batch = W.make_batch(W.TINY, 64, [40, 70], 10, 20, rng)
+    t = W.host_tensors(batch, rng)
+    bad = W.MixedBatch(**{**batch.__dict__})
+    bad.decode_pages = batch.decode_pages.copy()
+    bad.decode_pages[1] = batch.num_pages + 5
+    r = gpu.Runner(bad, t)
+    r.attend()
+    code, detail = r.status()
+    assert code == r.B.SW_ERR_OUT_OF_RANGE
+    assert r.status() == (0, 0)           # cleared by the read
+    bad2 = W.MixedBatch(**{**batch.__dict__})
+    bad2.prefill_pages = batch.prefill_pages.copy()
+    bad2.prefill_pages[-1] = -3
+    r2 = gpu.Runner(bad2, t)
+    r2.append()
+    assert r2.status()[0] == r2.B.SW_ERR_OUT_OF_RANGE
+    # a good iteration on the same context still works afterwards
+    run_and_compare(gpu, oracle, batch, t, what="after bad ids")
+
+
+def test_host_argument_errors(gpu):
+    from paper_2609_07883_b200 import binding as B
+
+    rng = np.random.default_rng(38)
+    batch = W.make_batch(W.TINY, 64, [40], 10, 20, rng)
+    t = W.host_tensors(batch, rng)
+    r = gpu.Runner(batch, t)
+    short = W.MixedBatch(**{**batch.__dict__})
+    short.prefill_pages = batch.prefill_pages[:-1].copy()
+    db = B.DeviceBatch(short, r.dev)
+    with pytest.raises(B.SwError) as e:
+        B.sw_mixed_attn_run(r.ctx, r.pool, db, r.q, r.out)
+    assert e.value.status == B.SW_ERR_OUT_OF_RANGE
+    big = W.make_batch(W.TINY, 64, [40], 10, 40, rng)   # chunk beyond the context's max_chunk
+    with pytest.raises(B.SwError) as e:
+        B.sw_mixed_attn_run(r.ctx, r.pool, B.DeviceBatch(big, r.dev), r.q, r.out)
+    assert e.value.status == B.SW_ERR_WORKSPACE
+
+
+def test_host_buffer_iteration_matches_device_path(gpu, oracle):
+    import torch
+
+    rng = np.random.default_rng(39)
+    batch = W.make_batch(W.AttnShape(8, 2, 128), 96, [100, 333, 17], 50, 60, rng)
+    t = W.host_tensors(batch, rng)
+    r = gpu.Runner(batch, t)
+    B = r.B
+    hs, keep = B.host_batch_struct(batch)
+    h_out = np.zeros_like(t["q"])
+    h_lse = np.zeros((batch.num_rows, batch.shape.num_q_heads), np.float32)
+    B.sw_mixed_iteration_host(r.ctx, r.pool, hs, t["q"], t["k_new"], t["v_new"], h_out, h_lse)
+    pool = t["pool"].copy()
+    oracle.kv_append(pool, batch, t["k_new"], t["v_new"])
+    assert np.array_equal(gpu.torch_to_bits(r.pool), pool)
+    ref, ref_lse, _ = oracle.mixed_attention(pool, batch, t["q"])
+    gpu.compare(W.bf16_bits_to_f64(h_out).reshape(-1, 128), h_lse.reshape(-1).astype(np.float64), ref, ref_lse, "host path")
+
+
+def test_chat_workload_sampled_rows(gpu, oracle):
+    rng = W.rng_for(1)
+    batch = W.chat_batch(n=16, chunk_len=128, rng=rng)
+    t = W.host_tensors(batch, rng)
+    C, n, Hq = batch.chunk_len, batch.num_decode, batch.shape.num_q_heads
+    rows = [0, 1, 15, 16, 17, 31, 32, 63, 64, 127] + [C + i for i in range(n)]
+    prs = np.random.default_rng(5)
+    pairs = [(r_, int(prs.integers(0, Hq))) for r_ in rows] + [(r_, int(prs.integers(0, Hq))) for r_ in rows]
+    run_and_compare(gpu, oracle, batch, t, pairs=pairs, what="chat n=16 C=128")
