@@ -76,7 +76,7 @@ struct sw_ctx {
     };
     std::vector<MapEntry> kv_maps;  // small cache: one entry per pool of a layer stack
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-    int bringup_prefill_rows = 1;
+    int bringup_prefill_rows = 0;
 };
 
 namespace {
@@ -264,7 +264,20 @@ sw_status sw_mixed_attn_run(sw_ctx* ctx, const void* kv_pool, const sw_batch* ba
     p.max_items = ctx->w.max_items;
     p.target_items = sw::kTargetItems;
     p.prefill_rows_on_decode_path = ctx->bringup_prefill_rows;
-    SW_CUDA(sw::launch_mixed_attn(l.head_dim, *kv_map, p, ctx->num_sms, static_cast<cudaStream_t>(stream)));
+    // q as [row][head][element] restricted to the chunk rows: one box = 128 tile rows (token-major, the g heads of a
+    // KV head minor) x 64 elements; rows past the chunk read as zero
+    CUtensorMap q_map = *kv_map;
+    if (p.C > 0 && !p.prefill_rows_on_decode_path) {
+        const cuuint64_t dims[3] = {(cuuint64_t)l.head_dim, (cuuint64_t)l.num_q_heads, (cuuint64_t)p.C};
+        const cuuint64_t strides[2] = {(cuuint64_t)l.head_dim * 2, (cuuint64_t)l.num_q_heads * l.head_dim * 2};
+        const cuuint32_t box[3] = {64, (cuuint32_t)p.group, (cuuint32_t)(128 / p.group)};
+        const cuuint32_t elem_strides[3] = {1, 1, 1};
+        CUresult r = ctx->encode(&q_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box,
+                                 elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return sw_fail(SW_ERR_CUDA, "cuTensorMapEncodeTiled(q) failed with CUresult %d", (int)r);
+    }
+    SW_CUDA(sw::launch_mixed_attn(l.head_dim, *kv_map, q_map, p, ctx->num_sms, static_cast<cudaStream_t>(stream)));
     return SW_OK;
 }
 

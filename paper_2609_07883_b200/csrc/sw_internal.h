@@ -67,8 +67,8 @@ struct AppendParams {
 
 // launchers (sw_kernels.cu)
 cudaError_t launch_kv_append(const AppendParams& p, cudaStream_t stream);
-cudaError_t launch_mixed_attn(int head_dim, const CUtensorMap& kv_map, const MixedParams& p, int num_sms,
-                              cudaStream_t stream);
+cudaError_t launch_mixed_attn(int head_dim, const CUtensorMap& kv_map, const CUtensorMap& q_map, const MixedParams& p,
+                              int num_sms, cudaStream_t stream);
 cudaError_t configure_kernels(int head_dim);
 size_t mixed_attn_smem_bytes(int head_dim);
 

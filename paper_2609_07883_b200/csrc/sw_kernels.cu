@@ -95,8 +95,9 @@ struct Geo {
     static constexpr int kStageBytes = 2 * kHalves * kBlockBytes;  // K then V of one (page, kv head)
     static constexpr int kRingBytes = kWarps * kStages * kStageBytes;
     static constexpr int kBarOffset = kRingBytes;                              // kWarps*kStages mbarriers
-    static constexpr int kPlanOffset = kBarOffset + kWarps * kStages * 8;      // int32 unit_prefix[kMaxDecode+1]
-    static constexpr int kMiscOffset = kPlanOffset + (kMaxDecode + 1) * 4;     // scan scratch etc.
+    static constexpr int kPfBarOffset = kBarOffset + kWarps * kStages * 8;     // barriers of the prefill tiles
+    static constexpr int kPlanOffset = kPfBarOffset + 32 * 8;                  // int32 unit_prefix[kMaxDecode+1]
+    static constexpr int kMiscOffset = kPlanOffset + (kMaxDecode + 1) * 4 + 12; // scan scratch, TMEM base, abort flag
     static constexpr int kSmemBytes = kMiscOffset + 256;
 };
 
@@ -430,12 +431,18 @@ __device__ bool run_unit(const CUtensorMap* kv_map, const MixedParams& p, const 
     return true;
 }
 
+}  // namespace sw
+#include "sw_prefill.cuh"
+namespace sw {
+
 // ---------------------------------------------------------------------------------------------------------------
 // the persistent kernel
 // ---------------------------------------------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid_constant__ CUtensorMap kv_map,
+                                                                    const __grid_constant__ CUtensorMap q_map,
                                                                     const MixedParams p) {
+    static_assert(PfGeo<D>::kBytes <= Geo<D>::kRingBytes, "prefill tiles must fit the region shared with the decode ring");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -445,12 +452,41 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     int* unit_prefix = reinterpret_cast<int*>(smem + Geo<D>::kPlanOffset);
     int* scratch = reinterpret_cast<int*>(smem + Geo<D>::kMiscOffset);
 
+    const bool tensor_prefill = p.C > 0 && !p.prefill_rows_on_decode_path;
+    volatile int* misc = reinterpret_cast<volatile int*>(scratch + 32);  // [0] TMEM base, [1] abort flag
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&kv_map);
         for (int i = 0; i < kWarps * kStages; ++i) mbar_init(base + Geo<D>::kBarOffset + i * 8, 1);
+        if (tensor_prefill) {
+            tma_prefetch_desc(&q_map);
+            pf_init_barriers(base + Geo<D>::kPfBarOffset);
+        }
+        misc[0] = 0;
+        misc[1] = 0;
         fence_mbar_init();
     }
     __syncthreads();
+
+    // chunk-prefill tiles first (long, tensor-bound); the decode units below fill the tail
+    if (tensor_prefill) {
+        if (warp == 1) {
+            tmem_alloc(smem_u32(const_cast<int*>(&misc[0])), 512);
+            tmem_relinquish();
+        }
+        tc_fence_before_sync();
+        __syncthreads();
+        tc_fence_after_sync();
+        PfShared sh;
+        sh.smem = base;
+        sh.bars = base + Geo<D>::kPfBarOffset;
+        sh.tmem = (uint32_t)misc[0];
+        sh.abort_flag = &misc[1];
+        prefill_phase<D>(&kv_map, &q_map, p, sh);
+        tc_fence_before_sync();
+        __syncthreads();
+        if (warp == 1) tmem_dealloc(sh.tmem, 512);
+        __syncthreads();
+    }
 
     const Plan plan = make_plan(p, unit_prefix, scratch);
     if (plan.total_items > p.max_items + plan.prefill_items) {
@@ -535,13 +571,13 @@ cudaError_t configure_kernels(int head_dim) {
                                 (int)mixed_attn_smem_bytes(128));
 }
 
-cudaError_t launch_mixed_attn(int head_dim, const CUtensorMap& kv_map, const MixedParams& p, int num_sms,
-                              cudaStream_t stream) {
+cudaError_t launch_mixed_attn(int head_dim, const CUtensorMap& kv_map, const CUtensorMap& q_map, const MixedParams& p,
+                              int num_sms, cudaStream_t stream) {
     const size_t smem = mixed_attn_smem_bytes(head_dim);
     if (head_dim == 64)
-        sw_mixed_attn_kernel<64><<<num_sms, kThreads, smem, stream>>>(kv_map, p);
+        sw_mixed_attn_kernel<64><<<num_sms, kThreads, smem, stream>>>(kv_map, q_map, p);
     else
-        sw_mixed_attn_kernel<128><<<num_sms, kThreads, smem, stream>>>(kv_map, p);
+        sw_mixed_attn_kernel<128><<<num_sms, kThreads, smem, stream>>>(kv_map, q_map, p);
     return cudaGetLastError();
 }
 

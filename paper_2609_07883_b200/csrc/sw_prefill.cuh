@@ -1,0 +1,377 @@
+// Chunk-prefill attention tiles on the 5th-generation tensor cores (tcgen05 + TMEM), included by sw_kernels.cu.
+//
+// One work item = one KV head x 256 query rows (two 128-row tiles).  A tile's rows are (token, query head of the
+// group) pairs, token-major: row r <-> chunk token tok0 + r / g, head kvh*g + r % g, so all g query heads that
+// share the KV head ride on the same K/V tiles.  Per 128-key KV tile j:
+//     S_t = Q_t K_j^T          tcgen05.mma, A and B from shared memory (K-major, 128-byte swizzle), D in TMEM
+//     P_t = exp2(S_t - m)      4 warps per tile, one thread per row (TMEM lane), P written back to TMEM as bf16
+//     O_t += P_t V_j           tcgen05.mma, A from TMEM, B = V from shared memory (MN-major), D in TMEM
+// Roles: warp 0 lane 0 issues TMA (Q once per item, K/V pages into a 2-stage ring), warp 1 lane 0 issues every
+// MMA, warp 2 zeroes V rows past the end of the prompt (unwritten page slots), warps 4-7 / 8-11 run the online
+// softmax of tile 0 / 1.  All hand-offs are mbarriers; every wait is bounded.
+#pragma once
+
+namespace sw {
+
+template <int D>
+struct PfGeo {
+    static constexpr int kHalves = D / 64;
+    static constexpr int kHalfBytes = 128 * 128;                 // [128 rows][64 elements], 128-byte swizzle
+    static constexpr int kTileBytes = kHalves * kHalfBytes;      // one Q, K or V tile
+    static constexpr int kQOffset = 0;                           // Q tile t at t * kTileBytes
+    static constexpr int kKVOffset = 2 * kTileBytes;             // stage s: K at s * 2 * kTileBytes, then V
+    static constexpr int kBytes = kKVOffset + 2 * 2 * kTileBytes;
+    static constexpr int kPageBytes = kPageSize * 128;           // one page's rows inside a half
+};
+
+enum PfBar {
+    kBarQFull = 0, kBarKFull = 1, kBarVLanded = 3, kBarVFull = 5, kBarKEmpty = 7, kBarVEmpty = 9,
+    kBarSFull = 11, kBarPFull = 13, kBarODone = 15, kPfBars = 17
+};
+
+struct PfShared {
+    uint32_t smem;    // 1024-aligned shared address of the tile region
+    uint32_t bars;    // shared address of the kPfBars mbarriers
+    uint32_t tmem;    // TMEM base (lane 0, column 0 of the 512-column allocation)
+    volatile int* abort_flag;
+};
+
+__device__ __forceinline__ void pf_init_barriers(uint32_t bars) {
+    for (int i = 0; i < kPfBars; ++i) mbar_init(bars + i * 8, (i == kBarPFull || i == kBarPFull + 1) ? 128 : 1);
+}
+
+// Bounded wait that also gives up when another role of this CTA has given up.
+__device__ __forceinline__ bool pf_wait(const PfShared& sh, int bar, uint32_t parity, int32_t* ctrl, int where) {
+    const uint32_t addr = sh.bars + bar * 8;
+    if (mbar_try_wait(addr, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t i = 0;; ++i) {
+        if (mbar_try_wait(addr, parity)) return true;
+        if ((i & 63) == 63) {
+            if (*sh.abort_flag) return false;
+            if (clock64() - t0 > kWaitBudgetCycles) break;
+        }
+    }
+    *sh.abort_flag = 1;
+    report(ctrl, SW_ERR_DEVICE_TIMEOUT, kSiteWait, (where << 8) | bar);
+    return false;
+}
+
+struct PfItem {
+    int kvh;
+    int tok0[2];     // first chunk token of each tile
+    int nkv[2];      // KV tiles each tile attends (0 = tile inactive)
+    int nkv_max;
+};
+
+template <int D>
+__device__ __forceinline__ PfItem pf_item(const MixedParams& p, int item, int n_tp) {
+    PfItem it;
+    const int tt = 128 / p.group;  // tokens per tile
+    const int tp = n_tp - 1 - item / p.Hkv;  // longest (latest tokens) first
+    it.kvh = item % p.Hkv;
+    it.nkv_max = 0;
+    for (int t = 0; t < 2; ++t) {
+        it.tok0[t] = (tp * 2 + t) * tt;
+        if (it.tok0[t] < p.C) {
+            const int last = min(it.tok0[t] + tt, p.C) - 1;
+            it.nkv[t] = (p.P + last) / 128 + 1;
+        } else {
+            it.nkv[t] = 0;
+        }
+        it.nkv_max = max(it.nkv_max, it.nkv[t]);
+    }
+    return it;
+}
+
+// ---- role: TMA producer (one thread) ---------------------------------------------------------------------------
+template <int D>
+__device__ __forceinline__ bool pf_produce(const CUtensorMap* kv_map, const CUtensorMap* q_map, const MixedParams& p,
+                                           const PfShared& sh, const PfItem& it, uint32_t& kv_it) {
+    using G = PfGeo<D>;
+    const int tt = 128 / p.group;
+    // Q tiles (rows past the chunk are zero-filled by the tensor map's bounds)
+    int active = (it.nkv[0] > 0) + (it.nkv[1] > 0);
+    mbar_arrive_expect_tx(sh.bars + kBarQFull * 8, active * G::kTileBytes);
+    for (int t = 0; t < 2; ++t)
+        if (it.nkv[t] > 0)
+            for (int h = 0; h < G::kHalves; ++h)
+                tma_load_3d(sh.smem + G::kQOffset + t * G::kTileBytes + h * G::kHalfBytes, q_map, sh.bars + kBarQFull * 8,
+                            h * 64, it.kvh * p.group, it.tok0[t]);
+    (void)tt;
+    const int npages = (p.P + p.C + kPageSize - 1) / kPageSize;
+    for (int j = 0; j < it.nkv_max; ++j, ++kv_it) {
+        const uint32_t s = kv_it & 1, n = kv_it >> 1;
+        const int pg0 = j * 8;
+        const int nvp = min(8, npages - pg0);
+        int ids[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ids[i] = i < nvp ? p.prefill_pages[pg0 + i] : 0;
+        const uint32_t kdst = sh.smem + G::kKVOffset + s * 2 * G::kTileBytes;
+        const uint32_t vdst = kdst + G::kTileBytes;
+        if (!pf_wait(sh, kBarKEmpty + s, (n & 1) ^ 1, p.ctrl, 1)) return false;
+        mbar_arrive_expect_tx(sh.bars + (kBarKFull + s) * 8, nvp * G::kHalves * G::kPageBytes);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (i < nvp)
+                for (int h = 0; h < G::kHalves; ++h)
+                    tma_load_4d(kdst + h * G::kHalfBytes + i * G::kPageBytes, kv_map, sh.bars + (kBarKFull + s) * 8, h * 64, 0,
+                                it.kvh, ids[i]);
+        if (!pf_wait(sh, kBarVEmpty + s, (n & 1) ^ 1, p.ctrl, 2)) return false;
+        mbar_arrive_expect_tx(sh.bars + (kBarVLanded + s) * 8, nvp * G::kHalves * G::kPageBytes);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (i < nvp)
+                for (int h = 0; h < G::kHalves; ++h)
+                    tma_load_4d(vdst + h * G::kHalfBytes + i * G::kPageBytes, kv_map, sh.bars + (kBarVLanded + s) * 8, h * 64,
+                                0, p.Hkv + it.kvh, ids[i]);
+    }
+    return true;
+}
+
+// ---- role: V sanitizer (one warp) -------------------------------------------------------------------------------
+// Keys at or past P + C are never attended, but their V rows still enter the P V product with weight zero; zero them
+// so that whatever an unwritten page slot (or a stale buffer) holds cannot turn 0 * x into NaN.
+template <int D>
+__device__ __forceinline__ bool pf_sanitize(const MixedParams& p, const PfShared& sh, const PfItem& it, uint32_t& kv_it) {
+    using G = PfGeo<D>;
+    const int lane = threadIdx.x & 31;
+    const int kv_total = p.P + p.C;
+    for (int j = 0; j < it.nkv_max; ++j, ++kv_it) {
+        const uint32_t s = kv_it & 1, n = kv_it >> 1;
+        if (!pf_wait(sh, kBarVLanded + s, n & 1, p.ctrl, 3)) return false;
+        const int first_dead = max(0, kv_total - j * 128);
+        if (first_dead < 128) {
+            const uint32_t vdst = sh.smem + G::kKVOffset + s * 2 * G::kTileBytes + G::kTileBytes;
+            const int chunks = (128 - first_dead) * 8;  // 16-byte pieces per half
+            for (int h = 0; h < G::kHalves; ++h)
+                for (int c = lane; c < chunks; c += 32) {
+                    const uint32_t addr = vdst + h * G::kHalfBytes + (first_dead + c / 8) * 128 + (c % 8) * 16;
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
+                }
+            fence_proxy_async_smem();
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(sh.bars + (kBarVFull + s) * 8);
+    }
+    return true;
+}
+
+// ---- role: MMA issuer (one thread) ------------------------------------------------------------------------------
+struct PfMmaState {
+    uint32_t kv_it = 0, q_it = 0;
+    uint32_t p_cnt[2] = {0, 0};
+};
+
+template <int D>
+__device__ __forceinline__ void pf_issue_qk(const PfShared& sh, int t, uint32_t s) {
+    using G = PfGeo<D>;
+    constexpr uint32_t idesc = umma_idesc_bf16(128, 128, 0, 0);
+    const uint32_t q = sh.smem + G::kQOffset + t * G::kTileBytes;
+    const uint32_t k = sh.smem + G::kKVOffset + s * 2 * G::kTileBytes;
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+        const uint32_t off = (ks >> 2) * G::kHalfBytes + (ks & 3) * 32;
+        tc_mma_ss(sh.tmem + t * 128, umma_desc_sw128(q + off, 16, 1024), umma_desc_sw128(k + off, 16, 1024), idesc, ks > 0);
+    }
+    tc_commit(sh.bars + (kBarSFull + t) * 8);
+}
+
+template <int D>
+__device__ __forceinline__ void pf_issue_pv(const PfShared& sh, int t, uint32_t s, bool first) {
+    using G = PfGeo<D>;
+    constexpr uint32_t idesc = umma_idesc_bf16(128, D, 0, 1);  // B = V is MN-major: [key][d] with d contiguous
+    const uint32_t v = sh.smem + G::kKVOffset + s * 2 * G::kTileBytes + G::kTileBytes;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks)  // 16 keys per instruction
+        tc_mma_ts(sh.tmem + 256 + t * D, sh.tmem + t * 128 + ks * 8, umma_desc_sw128(v + ks * 2 * 1024, G::kHalfBytes, 1024),
+                  idesc, !(first && ks == 0));
+    tc_commit(sh.bars + (kBarODone + t) * 8);
+}
+
+template <int D>
+__device__ __forceinline__ bool pf_mma(const MixedParams& p, const PfShared& sh, const PfItem& it, PfMmaState& st) {
+    auto act = [&](int t, int j) { return j < it.nkv[t]; };
+    auto last_active = [&](int j) { return act(1, j) ? 1 : 0; };
+    if (!pf_wait(sh, kBarQFull, st.q_it & 1, p.ctrl, 4)) return false;
+    {
+        const uint32_t s = st.kv_it & 1, n = st.kv_it >> 1;
+        if (!pf_wait(sh, kBarKFull + s, n & 1, p.ctrl, 5)) return false;
+        tc_fence_after_sync();
+        for (int t = 0; t < 2; ++t)
+            if (act(t, 0)) pf_issue_qk<D>(sh, t, s);
+        tc_commit(sh.bars + (kBarKEmpty + s) * 8);
+    }
+    for (int j = 0; j < it.nkv_max; ++j) {
+        const uint32_t cur = st.kv_it + j;
+        const uint32_t s = cur & 1, n = cur >> 1;
+        if (!pf_wait(sh, kBarVFull + s, n & 1, p.ctrl, 6)) return false;
+        const bool more = j + 1 < it.nkv_max;
+        if (more && !pf_wait(sh, kBarKFull + (s ^ 1), ((cur + 1) >> 1) & 1, p.ctrl, 7)) return false;
+        for (int t = 0; t < 2; ++t) {
+            if (act(t, j)) {
+                if (!pf_wait(sh, kBarPFull + t, st.p_cnt[t] & 1, p.ctrl, 8)) return false;
+                st.p_cnt[t] += 1;
+                tc_fence_after_sync();
+                pf_issue_pv<D>(sh, t, s, j == 0);
+            }
+            if (t == last_active(j)) tc_commit(sh.bars + (kBarVEmpty + s) * 8);
+            if (act(t, j + 1)) pf_issue_qk<D>(sh, t, s ^ 1);
+            if (more && t == last_active(j + 1)) tc_commit(sh.bars + (kBarKEmpty + (s ^ 1)) * 8);
+        }
+    }
+    st.kv_it += it.nkv_max;
+    st.q_it += 1;
+    return true;
+}
+
+// ---- role: online softmax + epilogue (4 warps per tile, one thread per row) ---------------------------------------
+struct PfSoftmaxState {
+    uint32_t s_cnt = 0, o_cnt = 0;  // completions of this tile's S-ready / O-updated barriers consumed so far
+};
+
+template <int D>
+__device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared& sh, const PfItem& it, int t,
+                                           PfSoftmaxState& st) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nkv = it.nkv[t];
+    if (nkv == 0) return true;
+    const int row = (warp & 3) * 32 + lane;
+    const int tok = it.tok0[t] + row / p.group;
+    const int head = it.kvh * p.group + row % p.group;
+    const int pos = p.P + tok;
+    const uint32_t lane_addr = sh.tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t s_addr = lane_addr + t * 128;  // P (bf16) aliases the first 64 columns of S
+    const uint32_t o_addr = lane_addr + 256 + t * D;
+    const float sl2 = p.sm_scale_log2;
+    float m_ref = -INFINITY, l_sum = 0.f;
+    uint32_t v[32];
+
+    for (int j = 0; j < nkv; ++j) {
+        if (!pf_wait(sh, kBarSFull + t, st.s_cnt & 1, p.ctrl, 9)) return false;
+        st.s_cnt += 1;
+        tc_fence_after_sync();
+        const int limit = pos - j * 128 + 1;  // columns [0, limit) are attended
+        const bool masked = limit < 128;
+        // pass 1: row maximum
+        float mx = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            tmem_ld_32x32b_x32(s_addr + c * 32, v);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float x = __uint_as_float(v[i]);
+                mx = (!masked || c * 32 + i < limit) ? fmaxf(mx, x) : mx;
+            }
+        }
+        const float m_new = fmaxf(m_ref, mx * sl2);
+        if (j == 0) {
+            m_ref = m_new;
+        } else {
+            // lazy rescale: keep the old reference unless some row's maximum grew by more than 2^8
+            const bool need = m_new - m_ref > 8.0f;
+            if (__any_sync(0xffffffffu, need)) {
+                if (!pf_wait(sh, kBarODone + t, (st.o_cnt + j - 1) & 1, p.ctrl, 10)) return false;
+                tc_fence_after_sync();
+                const float f = need ? fast_exp2(m_ref - m_new) : 1.f;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    tmem_ld_32x32b_x32(o_addr + c * 32, v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * f);
+                    tmem_st_32x32b_x32(o_addr + c * 32, v);
+                }
+                tc_wait_st();
+                if (need) {
+                    l_sum *= f;
+                    m_ref = m_new;
+                }
+            }
+        }
+        // pass 2: P = exp2(S * scale - m_ref), packed to bf16 over the columns of S already read
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            tmem_ld_32x32b_x32(s_addr + c * 32, v);
+            tc_wait_ld();
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                float p0 = fast_exp2(fmaf(__uint_as_float(v[2 * i]), sl2, -m_ref));
+                float p1 = fast_exp2(fmaf(__uint_as_float(v[2 * i + 1]), sl2, -m_ref));
+                if (masked) {
+                    p0 = (c * 32 + 2 * i < limit) ? p0 : 0.f;
+                    p1 = (c * 32 + 2 * i + 1 < limit) ? p1 : 0.f;
+                }
+                l_sum += p0 + p1;
+                pk[i] = pack_bf16x2(p0, p1);
+            }
+            tmem_st_32x32b_x16(s_addr + c * 16, pk);
+        }
+        tc_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive(sh.bars + (kBarPFull + t) * 8);
+    }
+
+    // epilogue: O / l -> bf16 -> out
+    if (!pf_wait(sh, kBarODone + t, (st.o_cnt + nkv - 1) & 1, p.ctrl, 11)) return false;
+    st.o_cnt += nkv;
+    tc_fence_after_sync();
+    const float inv = 1.f / l_sum;
+    const bool row_ok = tok < p.C;
+    __nv_bfloat16* dst = p.out + ((int64_t)tok * p.Hq + head) * D;
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) {
+        tmem_ld_32x32b_x32(o_addr + c * 32, v);
+        tc_wait_ld();
+        if (row_ok) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint4 w;
+                w.x = pack_bf16x2(__uint_as_float(v[8 * i + 0]) * inv, __uint_as_float(v[8 * i + 1]) * inv);
+                w.y = pack_bf16x2(__uint_as_float(v[8 * i + 2]) * inv, __uint_as_float(v[8 * i + 3]) * inv);
+                w.z = pack_bf16x2(__uint_as_float(v[8 * i + 4]) * inv, __uint_as_float(v[8 * i + 5]) * inv);
+                w.w = pack_bf16x2(__uint_as_float(v[8 * i + 6]) * inv, __uint_as_float(v[8 * i + 7]) * inv);
+                *reinterpret_cast<uint4*>(dst + c * 32 + i * 8) = w;
+            }
+        }
+    }
+    if (row_ok && p.lse) p.lse[(int64_t)tok * p.Hq + head] = (m_ref + __log2f(l_sum)) * 0.6931471805599453f;
+    tc_fence_before_sync();
+    return true;
+}
+
+// ---- the prefill phase of one CTA ----------------------------------------------------------------------------------
+template <int D>
+__device__ __forceinline__ void prefill_phase(const CUtensorMap* kv_map, const CUtensorMap* q_map, const MixedParams& p,
+                                              const PfShared& sh) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tok_per_item = 256 / p.group;
+    const int n_tp = (p.C + tok_per_item - 1) / tok_per_item;
+    const int n_items = n_tp * p.Hkv;
+    uint32_t prod_kv_it = 0, san_kv_it = 0;
+    PfMmaState mma_state;
+    PfSoftmaxState sm_state;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const PfItem it = pf_item<D>(p, item, n_tp);
+        bool ok = true;
+        if (warp == 0) {
+            if (lane == 0) ok = pf_produce<D>(kv_map, q_map, p, sh, it, prod_kv_it);
+        } else if (warp == 1) {
+            if (lane == 0) ok = pf_mma<D>(p, sh, it, mma_state);
+        } else if (warp == 2) {
+            ok = pf_sanitize<D>(p, sh, it, san_kv_it);
+        } else if (warp >= 4) {
+            ok = pf_softmax<D>(p, sh, it, (warp - 4) >> 2, sm_state);
+        }
+        (void)ok;
+        __syncwarp();
+        tc_fence_before_sync();
+        __syncthreads();
+        tc_fence_after_sync();
+        if (*sh.abort_flag) break;
+    }
+}
+
+}  // namespace sw
