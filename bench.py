@@ -63,9 +63,21 @@ def attention_work(batch: W.MixedBatch) -> dict:
     }
 
 
+WORKLOAD_DEFAULTS = {  # decodes, chunk, prefix
+    "chat": (64, 512, 512),
+    "mixed": (128, 4096, 28672),
+    "long": (16, 4096, 98304),
+}
+
+
 def make_workload(args, rank: int) -> W.MixedBatch:
-    rng = W.rng_for(1, salt=rank)
-    return W.chat_batch(n=args.decodes, chunk_len=args.chunk, prefix_len=args.prefix, rng=rng)
+    """chat: contexts U[256, 2048]; mixed: lognormal(median 2048, sigma 1) clipped to [128, 16384];
+    long: U[32768, 131072].  The pool holds the live pages plus a little slack."""
+    if args.workload == "chat":
+        return W.chat_batch(n=args.decodes, chunk_len=args.chunk, prefix_len=args.prefix, rng=W.rng_for(1, salt=rank))
+    if args.workload == "mixed":
+        return W.mixed_batch(args.chunk, args.prefix, n=args.decodes, rng=W.rng_for(2, salt=rank))
+    return W.long_batch(args.chunk, args.prefix, n=args.decodes, rng=W.rng_for(3, salt=rank))
 
 
 # ---------------------------------------------------------------------------------------------------------------
@@ -184,8 +196,10 @@ def run_reference(args) -> dict:
 
 
 def workload_config(args, batch) -> dict:
-    return {"workload": f"chat-like iteration, Llama-3-8B attention shape 32/8/128 bf16, 16-token pages: {args.decodes} decodes "
-                        f"with contexts U[256,2048] (total {batch.total_decode_ctx} tokens) + prefill chunk C={args.chunk} at "
+    dist = {"chat": "U[256,2048]", "mixed": "lognormal(median 2048, sigma 1) clipped to [128,16384]",
+            "long": "U[32768,131072]"}[args.workload]
+    return {"workload": f"{args.workload} iteration, Llama-3-8B attention shape 32/8/128 bf16, 16-token pages: {args.decodes} decodes "
+                        f"with contexts {dist} (total {batch.total_decode_ctx} tokens) + prefill chunk C={args.chunk} at "
                         f"prefix {args.prefix}",
             "layers_rotated": args.layers, "l2": "inputs larger than L2: step k uses pool k mod layers",
             "decodes": args.decodes, "chunk": args.chunk, "prefix": args.prefix}
@@ -331,14 +345,21 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--decodes", type=int, default=64)
-    ap.add_argument("--chunk", type=int, default=512)
-    ap.add_argument("--prefix", type=int, default=512)
-    ap.add_argument("--layers", type=int, default=8, help="pools rotated through (working set > L2)")
+    ap.add_argument("--workload", default="chat", choices=sorted(WORKLOAD_DEFAULTS))
+    ap.add_argument("--decodes", type=int, default=None)
+    ap.add_argument("--chunk", type=int, default=None)
+    ap.add_argument("--prefix", type=int, default=None)
+    ap.add_argument("--layers", type=int, default=None, help="pools rotated through (working set > L2)")
     ap.add_argument("--cpu-budget-keys", type=int, default=1_000_000_000)
     ap.add_argument("--ref-budget-keys", type=int, default=1_000_000_000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    dn, dc, dp = WORKLOAD_DEFAULTS[args.workload]
+    args.decodes = dn if args.decodes is None else args.decodes
+    args.chunk = dc if args.chunk is None else args.chunk
+    args.prefix = dp if args.prefix is None else args.prefix
+    if args.layers is None:
+        args.layers = 8 if args.workload == "chat" else 2
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     res = run_reference(args) if args.impl == "reference" else run_ours(args)
     if res:
