@@ -452,7 +452,8 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     int* unit_prefix = reinterpret_cast<int*>(smem + Geo<D>::kPlanOffset);
     int* scratch = reinterpret_cast<int*>(smem + Geo<D>::kMiscOffset);
 
-    const bool tensor_prefill = p.C > 0 && !p.prefill_rows_on_decode_path;
+    // CTAs beyond the number of prefill items skip the tensor phase altogether (no TMEM, no register re-budgeting)
+    const bool tensor_prefill = p.C > 0 && !p.prefill_rows_on_decode_path && (int)blockIdx.x < pf_num_items(p);
     volatile int* misc = reinterpret_cast<volatile int*>(scratch + 32);  // [0] TMEM base, [1] abort flag
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&kv_map);

@@ -29,6 +29,9 @@ enum PfBar {
     kBarSFull = 11, kBarPFull = 13, kBarODone = 15, kPfBars = 17
 };
 
+// register budgets per warpgroup during the prefill phase: 128 * 72 + 256 * 216 <= 384 * 168
+constexpr int kPfRegsLaunch = 168, kPfRegsLight = 72, kPfRegsHeavy = 216;
+
 struct PfShared {
     uint32_t smem;    // 1024-aligned shared address of the tile region
     uint32_t bars;    // shared address of the kPfBars mbarriers
@@ -55,6 +58,12 @@ __device__ __forceinline__ bool pf_wait(const PfShared& sh, int bar, uint32_t pa
     *sh.abort_flag = 1;
     report(ctrl, SW_ERR_DEVICE_TIMEOUT, kSiteWait, (where << 8) | bar);
     return false;
+}
+
+// number of (256-row tile pair, kv head) work items of the chunk
+__device__ __forceinline__ int pf_num_items(const MixedParams& p) {
+    const int tok_per_item = 256 / p.group;
+    return ((p.C + tok_per_item - 1) / tok_per_item) * p.Hkv;
 }
 
 struct PfItem {
@@ -226,6 +235,25 @@ __device__ __forceinline__ bool pf_mma(const MixedParams& p, const PfShared& sh,
 }
 
 // ---- role: online softmax + epilogue (4 warps per tile, one thread per row) ---------------------------------------
+// exp2 either on the special-function unit or, for a fixed share of the elements, as a cubic on the FMA pipe
+// (round to nearest integer with the 1.5 * 2^23 trick, minimax cubic of 2^f on [-0.5, 0.5], relative error 7.5e-5 —
+// far below the bf16 rounding of P — exponent added as integer bits).  The two pipes then share the row's 128 exps.
+constexpr int kPolyEvery = 0;  // every kPolyEvery-th pair computes its first element with the polynomial; 0 = never
+template <bool kPoly>
+__device__ __forceinline__ float pf_exp2(float x) {
+    if constexpr (!kPoly) {
+        return fast_exp2(x);
+    } else {
+        x = fmaxf(x, -126.f);
+        const float t = x + 12582912.f;
+        const float f = x - (t - 12582912.f);
+        float r = fmaf(f, 0.0551716648f, 0.2426111251f);
+        r = fmaf(r, f, 0.6932609677f);
+        r = fmaf(r, f, 0.9999280572f);
+        return __int_as_float(__float_as_int(r) + (__float_as_int(t) << 23));
+    }
+}
+
 struct PfSoftmaxState {
     uint32_t s_cnt = 0, o_cnt = 0;  // completions of this tile's S-ready / O-updated barriers consumed so far
 };
@@ -251,20 +279,25 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
         if (!pf_wait(sh, kBarSFull + t, st.s_cnt & 1, p.ctrl, 9)) return false;
         st.s_cnt += 1;
         tc_fence_after_sync();
+        // the whole row of S (128 fp32) in registers: one TMEM read per element
+        uint32_t s[128];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x32(s_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+        tc_wait_ld();
         const int limit = pos - j * 128 + 1;  // columns [0, limit) are attended
-        const bool masked = limit < 128;
-        // pass 1: row maximum
-        float mx = -INFINITY;
+        if (limit < 128) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            tmem_ld_32x32b_x32(s_addr + c * 32, v);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const float x = __uint_as_float(v[i]);
-                mx = (!masked || c * 32 + i < limit) ? fmaxf(mx, x) : mx;
-            }
+            for (int i = 0; i < 128; ++i) s[i] = i < limit ? s[i] : 0xff800000u;  // -inf: exp2 gives exactly 0
         }
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 128; i += 4) {
+            mx0 = fmaxf(mx0, __uint_as_float(s[i]));
+            mx1 = fmaxf(mx1, __uint_as_float(s[i + 1]));
+            mx2 = fmaxf(mx2, __uint_as_float(s[i + 2]));
+            mx3 = fmaxf(mx3, __uint_as_float(s[i + 3]));
+        }
+        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
         const float m_new = fmaxf(m_ref, mx * sl2);
         if (j == 0) {
             m_ref = m_new;
@@ -290,25 +323,24 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
                 }
             }
         }
-        // pass 2: P = exp2(S * scale - m_ref), packed to bf16 over the columns of S already read
+        // P = exp2(S * scale - m_ref), packed to bf16 over the columns of S (all of S is already in registers)
+        const float neg_m = -m_ref;
+        float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            tmem_ld_32x32b_x32(s_addr + c * 32, v);
-            tc_wait_ld();
             uint32_t pk[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-                float p0 = fast_exp2(fmaf(__uint_as_float(v[2 * i]), sl2, -m_ref));
-                float p1 = fast_exp2(fmaf(__uint_as_float(v[2 * i + 1]), sl2, -m_ref));
-                if (masked) {
-                    p0 = (c * 32 + 2 * i < limit) ? p0 : 0.f;
-                    p1 = (c * 32 + 2 * i + 1 < limit) ? p1 : 0.f;
-                }
-                l_sum += p0 + p1;
+                const float p0 = pf_exp2<kPolyEvery != 0 && (i % (kPolyEvery ? kPolyEvery : 1)) == 0>(
+                    fmaf(__uint_as_float(s[c * 32 + 2 * i]), sl2, neg_m));
+                const float p1 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + 2 * i + 1]), sl2, neg_m));
+                sum0 += p0;
+                sum1 += p1;
                 pk[i] = pack_bf16x2(p0, p1);
             }
             tmem_st_32x32b_x16(s_addr + c * 16, pk);
         }
+        l_sum += sum0 + sum1;
         tc_wait_st();
         tc_fence_before_sync();
         mbar_arrive(sh.bars + (kBarPFull + t) * 8);
@@ -353,24 +385,38 @@ __device__ __forceinline__ void prefill_phase(const CUtensorMap* kv_map, const C
     uint32_t prod_kv_it = 0, san_kv_it = 0;
     PfMmaState mma_state;
     PfSoftmaxState sm_state;
-    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const PfItem it = pf_item<D>(p, item, n_tp);
-        bool ok = true;
-        if (warp == 0) {
-            if (lane == 0) ok = pf_produce<D>(kv_map, q_map, p, sh, it, prod_kv_it);
-        } else if (warp == 1) {
-            if (lane == 0) ok = pf_mma<D>(p, sh, it, mma_state);
-        } else if (warp == 2) {
-            ok = pf_sanitize<D>(p, sh, it, san_kv_it);
-        } else if (warp >= 4) {
-            ok = pf_softmax<D>(p, sh, it, (warp - 4) >> 2, sm_state);
-        }
-        (void)ok;
+    // The softmax warpgroups hold a whole row of S in registers; the TMA / MMA / sanitizer warps need few.  The two
+    // kinds of warps run separate loops (so that each gets its own register budget) and meet at a named barrier at
+    // the end of every item.
+    auto item_sync = [&]() {
         __syncwarp();
         tc_fence_before_sync();
-        __syncthreads();
+        named_barrier_sync(1, kThreads);
         tc_fence_after_sync();
-        if (*sh.abort_flag) break;
+        return *sh.abort_flag == 0;
+    };
+    if (warp < 4) {
+        setmaxnreg_dec<kPfRegsLight>();
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+            const PfItem it = pf_item<D>(p, item, n_tp);
+            if (warp == 0) {
+                if (lane == 0) pf_produce<D>(kv_map, q_map, p, sh, it, prod_kv_it);
+            } else if (warp == 1) {
+                if (lane == 0) pf_mma<D>(p, sh, it, mma_state);
+            } else if (warp == 2) {
+                pf_sanitize<D>(p, sh, it, san_kv_it);
+            }
+            if (!item_sync()) break;
+        }
+        setmaxnreg_inc<kPfRegsLaunch>();
+    } else {
+        setmaxnreg_inc<kPfRegsHeavy>();
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+            const PfItem it = pf_item<D>(p, item, n_tp);
+            pf_softmax<D>(p, sh, it, (warp - 4) >> 2, sm_state);
+            if (!item_sync()) break;
+        }
+        setmaxnreg_dec<kPfRegsLaunch>();
     }
 }
 

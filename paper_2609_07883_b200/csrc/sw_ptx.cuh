@@ -186,6 +186,22 @@ __device__ __forceinline__ void tmem_st_32x32b_x32(uint32_t taddr, const uint32_
         : "memory");
 }
 
+// Named barrier: every participating thread executes a bar.sync with the same id and thread count (they need not
+// be the same instruction, so differently specialised warps can meet here).
+__device__ __forceinline__ void named_barrier_sync(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// Per-warpgroup register budget (all four warps of the warpgroup execute it together).
+template <int kRegs>
+__device__ __forceinline__ void setmaxnreg_inc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegs));
+}
+template <int kRegs>
+__device__ __forceinline__ void setmaxnreg_dec() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs));
+}
+
 // Shared-memory matrix descriptor for tcgen05.mma, 128-byte swizzle, 16-byte units:
 //   bits [0,14) start address >> 4, [16,30) leading byte offset >> 4, [32,46) stride byte offset >> 4,
 //   [46,48) descriptor version (1 on sm_100), [61,64) layout type (2 = 128-byte swizzle).
