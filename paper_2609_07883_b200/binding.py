@@ -11,7 +11,10 @@ from pathlib import Path
 
 import numpy as np
 
-_LIB_PATH = Path(__file__).resolve().parent / "libsloweave.so"
+import os
+
+# SLOWEAVE_LIB overrides the library file (used to compare differently tuned builds of the same sources)
+_LIB_PATH = Path(os.environ.get("SLOWEAVE_LIB") or Path(__file__).resolve().parent / "libsloweave.so")
 if not _LIB_PATH.exists():
     raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2609_07883_b200.build` "
                       "(there is no CPU or library fallback)")

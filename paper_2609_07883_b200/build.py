@@ -22,15 +22,16 @@ def _stale() -> bool:
     return any(p.stat().st_mtime > t for p in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> Path:
+def build(force: bool = False, verbose: bool = False, defines=(), out: Path | None = None) -> Path:
     """Compile every source for sm_100a and link the shared library.  cudart is linked statically and the one
     driver function needed (tensor-map encode) is resolved at run time, so the library loads without a GPU."""
-    if not force and not _stale():
+    lib = Path(out) if out is not None else LIB
+    if out is None and not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    objdir = HERE / "build"
-    objdir.mkdir(exist_ok=True)
-    common = [nvcc, "-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "-I", str(INCLUDE), "-I", str(CSRC)] + ARCH
+    objdir = HERE / "build" / (lib.stem if out is not None else "default")
+    objdir.mkdir(parents=True, exist_ok=True)
+    common = [nvcc, "-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "-I", str(INCLUDE), "-I", str(CSRC)] + ARCH + [f"-D{d}" for d in defines]
     if verbose:
         common += ["-Xptxas", "-v"]
     objs = []
@@ -48,10 +49,10 @@ def build(force: bool = False, verbose: bool = False) -> Path:
         failed = failed or pr.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    tmp = LIB.with_suffix(f".{os.getpid()}.tmp")
+    tmp = lib.with_suffix(f".{os.getpid()}.tmp")
     subprocess.check_call([nvcc, "-shared", "-o", str(tmp)] + objs + ARCH + ["-cudart", "static"])
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":

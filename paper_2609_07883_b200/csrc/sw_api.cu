@@ -24,7 +24,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Offsets of the regions inside the caller's workspace.
 struct WsLayout {
-    size_t ctrl, tickets, part_ml, part_o, st_q, st_k, st_v, st_out, st_lse, st_pages, total;
+    size_t ctrl, tickets, part_ml, part_o, pf_tickets, pf_ml, pf_o, st_q, st_k, st_v, st_out, st_lse, st_pages, total;
     int max_items;
 };
 
@@ -49,6 +49,10 @@ WsLayout ws_layout(const sw_layout& l, int max_chunk, int max_decode, int64_t ma
     w.tickets = off;  off = align_up(off + (size_t)std::max(1, max_decode) * l.num_kv_heads * 4, 256);
     w.part_ml = off;  off = align_up(off + (size_t)w.max_items * 2 * sw::kMaxGroup * 4, 256);
     w.part_o = off;   off = align_up(off + (size_t)w.max_items * g * l.head_dim * 4, 256);
+    const size_t groups = ((size_t)max_chunk + (256 / g) - 1) / (256 / g);
+    w.pf_tickets = off; off = align_up(off + std::max<size_t>(1, groups) * l.num_kv_heads * 2 * 4, 256);
+    w.pf_ml = off;    off = align_up(off + (size_t)2 * sw::kMaxCtas * 2 * 256 * 4, 256);
+    w.pf_o = off;     off = align_up(off + (max_chunk > 0 ? (size_t)2 * sw::kMaxCtas * 2 * 128 * l.head_dim * 4 : 0), 256);
     w.st_q = off;     off = align_up(off + rows * l.num_q_heads * l.head_dim * 2, 256);
     w.st_k = off;     off = align_up(off + rows * l.num_kv_heads * l.head_dim * 2, 256);
     w.st_v = off;     off = align_up(off + rows * l.num_kv_heads * l.head_dim * 2, 256);
@@ -140,7 +144,7 @@ extern "C" {
 
 size_t sw_workspace_bytes(const sw_layout* layout, int32_t max_chunk, int32_t max_decode, int64_t max_pages) {
     if (!layout || !layout_supported(*layout) || max_chunk < 0 || max_decode < 0 || max_pages < 0 ||
-        max_decode > sw::kMaxDecode)
+        max_decode > sw::kMaxDecode || max_chunk > sw::kMaxChunk)
         return 0;
     return ws_layout(*layout, max_chunk, max_decode, max_pages).total;
 }
@@ -151,8 +155,9 @@ sw_status sw_create(const sw_layout* layout, int device, void* workspace, size_t
     if (!layout_supported(*layout))
         return sw_fail(SW_ERR_UNSUPPORTED,
                        "sw_create: supported shapes are head_dim 64|128, page_size 16, q/kv head ratio 1|2|4|8");
-    if (max_chunk < 0 || max_decode < 0 || max_pages < 0 || max_decode > sw::kMaxDecode)
-        return sw_fail(SW_ERR_INVALID_ARG, "sw_create: limits out of range (max_decode <= %d)", sw::kMaxDecode);
+    if (max_chunk < 0 || max_decode < 0 || max_pages < 0 || max_decode > sw::kMaxDecode || max_chunk > sw::kMaxChunk)
+        return sw_fail(SW_ERR_INVALID_ARG, "sw_create: limits out of range (max_decode <= %d, max_chunk <= %d)", sw::kMaxDecode,
+                       sw::kMaxChunk);
     const WsLayout w = ws_layout(*layout, max_chunk, max_decode, max_pages);
     if (!workspace || workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0)
         return sw_fail(SW_ERR_WORKSPACE, "sw_create: workspace must be 256-byte aligned and hold %zu bytes", w.total);
@@ -167,7 +172,7 @@ sw_status sw_create(const sw_layout* layout, int device, void* workspace, size_t
     ctx->layout = *layout;
     if (ctx->layout.sm_scale <= 0.f) ctx->layout.sm_scale = 1.0f / std::sqrt((float)layout->head_dim);
     ctx->device = device;
-    ctx->num_sms = prop.multiProcessorCount;
+    ctx->num_sms = std::min(prop.multiProcessorCount, sw::kMaxCtas);
     ctx->max_chunk = max_chunk;
     ctx->max_decode = max_decode;
     ctx->max_pages = max_pages;
@@ -181,7 +186,7 @@ sw_status sw_create(const sw_layout* layout, int device, void* workspace, size_t
         return sw_fail(SW_ERR_CUDA, "sw_create: cuTensorMapEncodeTiled is not available from the driver");
     }
     ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
-    e = cudaMemset(ctx->ws, 0, w.st_q);  // control words, tickets and partial-result scratch start at zero
+    e = cudaMemset(ctx->ws, 0, w.pf_ml);  // control words, tickets and split-KV scratch start at zero
     if (e == cudaSuccess) e = sw::configure_kernels(layout->head_dim);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
@@ -263,6 +268,9 @@ sw_status sw_mixed_attn_run(sw_ctx* ctx, const void* kv_pool, const sw_batch* ba
     p.part_o = reinterpret_cast<float*>(ctx->ws + ctx->w.part_o);
     p.max_items = ctx->w.max_items;
     p.target_items = sw::kTargetItems;
+    p.pf_ml = reinterpret_cast<float*>(ctx->ws + ctx->w.pf_ml);
+    p.pf_o = reinterpret_cast<float*>(ctx->ws + ctx->w.pf_o);
+    p.pf_tickets = reinterpret_cast<int32_t*>(ctx->ws + ctx->w.pf_tickets);
     p.prefill_rows_on_decode_path = ctx->bringup_prefill_rows;
     // q as [row][head][element] restricted to the chunk rows: one box = 128 tile rows (token-major, the g heads of a
     // KV head minor) x 64 elements; rows past the chunk read as zero

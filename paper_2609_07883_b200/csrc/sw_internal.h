@@ -16,6 +16,8 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kTargetItems = 4096;      // split-KV units aimed at per launch (bounds the partial-result scratch)
 constexpr int kMinSplitTokens = 256;    // never split a decode context finer than this
 constexpr int kMaxGroup = 8;            // query heads per KV head
+constexpr int kMaxCtas = 192;           // persistent CTAs (one per SM) the scratch is sized for
+constexpr int kMaxChunk = 65536;        // chunk tokens per iteration (256-row groups are planned in shared memory)
 
 // Control words at the start of the workspace.
 enum CtrlWord { kCtrWork = 0, kCtrDone = 1, kCtrStatus = 2, kCtrDetail = 3, kCtrWords = 64 };
@@ -47,6 +49,10 @@ struct MixedParams {
     float* part_o;      // [max_items][group * D]
     int max_items;      // partial-result slots available
     int target_items;   // split-KV units aimed at (<= max_items - n*Hkv)
+    // scratch of prefill items finished by several CTAs
+    float* pf_ml;        // [2 * kMaxCtas][2][2][128]
+    float* pf_o;         // [2 * kMaxCtas][2][128][D]
+    int32_t* pf_tickets; // [items][2]
     int prefill_rows_on_decode_path;  // bring-up switch: run every chunk row as a one-token unit
 };
 

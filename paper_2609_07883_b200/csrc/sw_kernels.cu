@@ -452,9 +452,8 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     int* unit_prefix = reinterpret_cast<int*>(smem + Geo<D>::kPlanOffset);
     int* scratch = reinterpret_cast<int*>(smem + Geo<D>::kMiscOffset);
 
-    // CTAs beyond the number of prefill items skip the tensor phase altogether (no TMEM, no register re-budgeting)
-    const bool tensor_prefill = p.C > 0 && !p.prefill_rows_on_decode_path && (int)blockIdx.x < pf_num_items(p);
-    volatile int* misc = reinterpret_cast<volatile int*>(scratch + 32);  // [0] TMEM base, [1] abort flag
+    const bool tensor_prefill = p.C > 0 && !p.prefill_rows_on_decode_path;
+    volatile int* misc = reinterpret_cast<volatile int*>(scratch + 32);  // [0] TMEM base, [1] abort flag, [2..3] ticket flags
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&kv_map);
         for (int i = 0; i < kWarps * kStages; ++i) mbar_init(base + Geo<D>::kBarOffset + i * 8, 1);
@@ -470,23 +469,31 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
 
     // chunk-prefill tiles first (long, tensor-bound); the decode units below fill the tail
     if (tensor_prefill) {
-        if (warp == 1) {
-            tmem_alloc(smem_u32(const_cast<int*>(&misc[0])), 512);
-            tmem_relinquish();
+        const PfPlan pplan = pf_make_plan(p, unit_prefix, scratch);
+        if ((int)blockIdx.x * pplan.spc < pplan.total_steps) {  // this CTA's range of steps is not empty
+            if (warp == 1) {
+                tmem_alloc(smem_u32(const_cast<int*>(&misc[0])), 512);
+                tmem_relinquish();
+            }
+            tc_fence_before_sync();
+            __syncthreads();
+            tc_fence_after_sync();
+            PfShared sh;
+            sh.smem = base;
+            sh.bars = base + Geo<D>::kPfBarOffset;
+            sh.tmem = (uint32_t)misc[0];
+            sh.abort_flag = &misc[1];
+            PfScratch scr;
+            scr.ml = p.pf_ml;
+            scr.o = p.pf_o;
+            scr.tickets = p.pf_tickets;
+            scr.flags = &misc[2];
+            prefill_phase<D>(&kv_map, &q_map, p, sh, pplan, scr);
+            tc_fence_before_sync();
+            __syncthreads();
+            if (warp == 1) tmem_dealloc(sh.tmem, 512);
         }
-        tc_fence_before_sync();
-        __syncthreads();
-        tc_fence_after_sync();
-        PfShared sh;
-        sh.smem = base;
-        sh.bars = base + Geo<D>::kPfBarOffset;
-        sh.tmem = (uint32_t)misc[0];
-        sh.abort_flag = &misc[1];
-        prefill_phase<D>(&kv_map, &q_map, p, sh);
-        tc_fence_before_sync();
-        __syncthreads();
-        if (warp == 1) tmem_dealloc(sh.tmem, 512);
-        __syncthreads();
+        __syncthreads();  // the plan's shared-memory array is reused by the decode plan
     }
 
     const Plan plan = make_plan(p, unit_prefix, scratch);
