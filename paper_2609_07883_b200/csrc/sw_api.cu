@@ -51,8 +51,8 @@ WsLayout ws_layout(const sw_layout& l, int max_chunk, int max_decode, int64_t ma
     w.part_o = off;   off = align_up(off + (size_t)w.max_items * g * l.head_dim * 4, 256);
     const size_t groups = ((size_t)max_chunk + (256 / g) - 1) / (256 / g);
     w.pf_tickets = off; off = align_up(off + std::max<size_t>(1, groups) * l.num_kv_heads * 2 * 4, 256);
-    w.pf_ml = off;    off = align_up(off + (size_t)2 * sw::kMaxCtas * 2 * 256 * 4, 256);
-    w.pf_o = off;     off = align_up(off + (max_chunk > 0 ? (size_t)2 * sw::kMaxCtas * 2 * 128 * l.head_dim * 4 : 0), 256);
+    w.pf_ml = off;    off = align_up(off + (size_t)sw::kMaxCtas * 2 * 256 * 4, 256);
+    w.pf_o = off;     off = align_up(off + (max_chunk > 0 ? (size_t)sw::kMaxCtas * 2 * 128 * l.head_dim * 4 : 0), 256);
     w.st_q = off;     off = align_up(off + rows * l.num_q_heads * l.head_dim * 2, 256);
     w.st_k = off;     off = align_up(off + rows * l.num_kv_heads * l.head_dim * 2, 256);
     w.st_v = off;     off = align_up(off + rows * l.num_kv_heads * l.head_dim * 2, 256);

@@ -20,7 +20,7 @@ constexpr int kMaxCtas = 192;           // persistent CTAs (one per SM) the scra
 constexpr int kMaxChunk = 65536;        // chunk tokens per iteration (256-row groups are planned in shared memory)
 
 // Control words at the start of the workspace.
-enum CtrlWord { kCtrWork = 0, kCtrDone = 1, kCtrStatus = 2, kCtrDetail = 3, kCtrWords = 64 };
+enum CtrlWord { kCtrWork = 0, kCtrDone = 1, kCtrStatus = 2, kCtrDetail = 3, kCtrPrefill = 4, kCtrWords = 64 };
 
 // Device-detected problem locators written to kCtrDetail (high byte = site, low 24 bits = index).
 enum DetailSite { kSiteAppendPage = 1, kSiteAppendLen = 2, kSiteAttnLen = 3, kSiteAttnPage = 4, kSiteWait = 5,
@@ -50,8 +50,8 @@ struct MixedParams {
     int max_items;      // partial-result slots available
     int target_items;   // split-KV units aimed at (<= max_items - n*Hkv)
     // scratch of prefill items finished by several CTAs
-    float* pf_ml;        // [2 * kMaxCtas][2][2][128]
-    float* pf_o;         // [2 * kMaxCtas][2][128][D]
+    float* pf_ml;        // [kMaxCtas][2][2][128]
+    float* pf_o;         // [kMaxCtas][2][128][D]
     int32_t* pf_tickets; // [items][2]
     int prefill_rows_on_decode_path;  // bring-up switch: run every chunk row as a one-token unit
 };

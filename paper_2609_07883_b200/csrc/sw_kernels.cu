@@ -469,8 +469,11 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
 
     // chunk-prefill tiles first (long, tensor-bound); the decode units below fill the tail
     if (tensor_prefill) {
-        const PfPlan pplan = pf_make_plan(p, unit_prefix, scratch);
-        if ((int)blockIdx.x * pplan.spc < pplan.total_steps) {  // this CTA's range of steps is not empty
+        const PfPlan pplan = pf_make_plan(p);
+        if (threadIdx.x == 0) misc[4] = atomicAdd(&p.ctrl[kCtrPrefill], 1);
+        __syncthreads();
+        const int first_entry = misc[4];
+        if (first_entry < pplan.n_entries) {  // CTA-uniform: this CTA has prefill work
             if (warp == 1) {
                 tmem_alloc(smem_u32(const_cast<int*>(&misc[0])), 512);
                 tmem_relinquish();
@@ -488,12 +491,12 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
             scr.o = p.pf_o;
             scr.tickets = p.pf_tickets;
             scr.flags = &misc[2];
-            prefill_phase<D>(&kv_map, &q_map, p, sh, pplan, scr);
+            prefill_phase<D>(&kv_map, &q_map, p, sh, pplan, scr, first_entry, &misc[5]);
             tc_fence_before_sync();
             __syncthreads();
             if (warp == 1) tmem_dealloc(sh.tmem, 512);
         }
-        __syncthreads();  // the plan's shared-memory array is reused by the decode plan
+        __syncthreads();
     }
 
     const Plan plan = make_plan(p, unit_prefix, scratch);
@@ -561,6 +564,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
         const int done = atomicAdd(&p.ctrl[kCtrDone], 1);
         if (done == (int)gridDim.x - 1) {
             p.ctrl[kCtrWork] = 0;
+            p.ctrl[kCtrPrefill] = 0;
             p.ctrl[kCtrDone] = 0;
             __threadfence();
         }

@@ -61,14 +61,23 @@ __device__ __forceinline__ bool pf_wait(const PfShared& sh, int bar, uint32_t pa
 }
 
 // ---- work decomposition -------------------------------------------------------------------------------------------
-// Items are ordered longest first: rank 0 is the last 256-row group of the chunk.  A "step" is one 128-key KV tile of
-// one item.  All steps of all items form one line of length W that is cut into equal ranges, one per CTA, so every
-// SM gets the same amount of tensor work whatever the chunk and prefix lengths are; an item cut by a range boundary
-// is finished by several CTAs, each writing a partial (m, l, O) for its piece, and the last one to arrive merges.
+// Items (one KV head x 256 query rows) are ordered longest first: rank 0 is the last 256-row group of the chunk.
+// A "step" is one 128-key KV tile of one item.  CTAs pull entries from a global counter.  The first n_whole
+// entries are whole items; the remaining r = n_items mod gridDim items (all of them when there are fewer items than
+// CTAs) would leave most SMs idle in the last wave, so each of them is cut along the KV axis into k pieces that run
+// side by side; every piece publishes a partial (m, l, O) and the last piece of an item to arrive merges them.
+// CTAs working at the same time thus stay at similar KV positions (their K/V tiles meet in L2).
+#ifndef SW_PF_MIN_PIECE_STEPS
+#define SW_PF_MIN_PIECE_STEPS 4
+#endif
+constexpr int kPfMinPieceSteps = SW_PF_MIN_PIECE_STEPS;
+
 struct PfPlan {
     int n_tp;           // 256-row groups of the chunk
-    int total_steps;    // W
-    int spc;            // steps per CTA (ceil(W / gridDim))
+    int n_items;        // n_tp * Hkv
+    int n_whole;        // entries [0, n_whole) are whole items
+    int pieces;         // k: pieces per tail item (1 = tail items are whole too)
+    int n_entries;      // n_whole + (n_items - n_whole) * k
     const int* prefix;  // shared memory [n_tp + 1]: steps of one kv head's items before rank r
 };
 
@@ -77,8 +86,10 @@ struct PfItem {
     int kvh;
     int tok0[2];     // first chunk token of each tile
     int nkv[2];      // KV tiles each tile attends in total (0 = tile has no rows)
-    int start;       // index of the item's step 0 on the line of all steps
-    int j0, j1;      // this CTA's piece of the item: KV tiles [j0, j1)
+    int nk;          // steps of the item = max(nkv)
+    int j0, j1;      // this entry's piece of the item: KV tiles [j0, j1)
+    int piece;       // index of the piece (0 when the item is whole)
+    int slot0;       // scratch slot of the item's piece 0 (tail items only)
 };
 
 __device__ __forceinline__ int pf_tiles_of(const MixedParams& p, int tok0) {
@@ -96,52 +107,59 @@ __device__ __forceinline__ int pf_steps_of_rank(const MixedParams& p, int n_tp, 
     const int tp = n_tp - 1 - r;
     return max(pf_tiles_of(p, (tp * 2) * tt), pf_tiles_of(p, (tp * 2 + 1) * tt));
 }
+// first KV tile of piece i when nk steps are cut into k pieces
+__device__ __forceinline__ int pf_piece_begin(int nk, int k, int i) { return (int)(((long long)nk * i) / k); }
 
-// Built by all threads of the CTA; `prefix` needs n_tp + 1 ints, `scratch` kWarps + 1 ints.
-__device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p, int* prefix, int* scratch) {
+__device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p) {
     PfPlan plan;
+    const int G = (int)gridDim.x;
     plan.n_tp = pf_num_groups(p);
-    const int per_thread = (plan.n_tp + kThreads - 1) / kThreads;
-    const int beg = min(plan.n_tp, (int)threadIdx.x * per_thread);
-    const int end = min(plan.n_tp, beg + per_thread);
-    int local = 0;
-    for (int r = beg; r < end; ++r) local += pf_steps_of_rank(p, plan.n_tp, r);
-    int total = 0;
-    int run = block_exclusive_scan(local, scratch, &total);
-    for (int r = beg; r < end; ++r) {
-        prefix[r] = run;
-        run += pf_steps_of_rank(p, plan.n_tp, r);
+    plan.n_items = plan.n_tp * p.Hkv;
+    const int r = plan.n_items % G;
+    plan.n_whole = plan.n_items - r;
+    plan.pieces = 1;
+    if (r > 0) {
+        // the tail items are the shortest ones; size the pieces by the shortest of them
+        // A piece costs its steps plus a merge that grows with k (about six steps' worth per piece merged), so
+        // k ~ sqrt(steps / 6); never more pieces than fit side by side, never pieces shorter than the minimum.
+        const int shortest = pf_steps_of_rank(p, plan.n_tp, plan.n_tp - 1);
+        int k = 1;
+        while ((k + 1) * (k + 1) * 6 <= shortest) ++k;
+        plan.pieces = max(1, min(min(G / r, k), shortest / kPfMinPieceSteps));
     }
-    if (threadIdx.x == 0) prefix[plan.n_tp] = total;
-    __syncthreads();
-    plan.total_steps = total * p.Hkv;
-    plan.spc = (plan.total_steps + (int)gridDim.x - 1) / (int)gridDim.x;
-    plan.prefix = prefix;
+    if (plan.pieces == 1) plan.n_whole = plan.n_items;
+    plan.n_entries = plan.n_whole + (plan.n_items - plan.n_whole) * plan.pieces;
+    plan.prefix = nullptr;
     return plan;
 }
 
-// The piece of the step line [x, range_end) that belongs to the item containing step x.
-__device__ __forceinline__ PfItem pf_locate(const MixedParams& p, const PfPlan& plan, int x, int range_end) {
-    int lo = 0, hi = plan.n_tp;  // largest rank with prefix[rank] * Hkv <= x
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (plan.prefix[mid] * p.Hkv <= x) lo = mid; else hi = mid;
-    }
-    const int rank = lo;
-    const int nk = plan.prefix[rank + 1] - plan.prefix[rank];
-    const int base = plan.prefix[rank] * p.Hkv;
+__device__ __forceinline__ PfItem pf_entry(const MixedParams& p, const PfPlan& plan, int entry) {
     PfItem it;
-    it.kvh = (x - base) / nk;
-    it.item = rank * p.Hkv + it.kvh;
-    it.start = base + it.kvh * nk;
+    if (entry < plan.n_whole) {
+        it.item = entry;
+        it.piece = 0;
+    } else {
+        it.item = plan.n_whole + (entry - plan.n_whole) / plan.pieces;
+        it.piece = (entry - plan.n_whole) % plan.pieces;
+    }
+    const int rank = it.item / p.Hkv;
+    it.kvh = it.item % p.Hkv;
     const int tt = 128 / p.group;
     const int tp = plan.n_tp - 1 - rank;
     for (int t = 0; t < 2; ++t) {
         it.tok0[t] = (tp * 2 + t) * tt;
         it.nkv[t] = pf_tiles_of(p, it.tok0[t]);
     }
-    it.j0 = x - it.start;
-    it.j1 = min(nk, range_end - it.start);
+    it.nk = max(it.nkv[0], it.nkv[1]);
+    if (entry < plan.n_whole) {
+        it.j0 = 0;
+        it.j1 = it.nk;
+        it.slot0 = 0;
+    } else {
+        it.j0 = pf_piece_begin(it.nk, plan.pieces, it.piece);
+        it.j1 = pf_piece_begin(it.nk, plan.pieces, it.piece + 1);
+        it.slot0 = (it.item - plan.n_whole) * plan.pieces;
+    }
     return it;
 }
 
@@ -316,8 +334,8 @@ struct PfSoftmaxState {
     uint32_t s_cnt = 0, o_cnt = 0;  // completions of this tile's S-ready / O-updated barriers consumed so far
 };
 
-// Scratch for items finished by several CTAs.  Slot = 2 * CTA + (0: the CTA's range starts inside the item,
-// 1: the item starts inside the CTA's range); per slot and tile: m[128], l[128] and O[128][D], all fp32.
+// Scratch for the tail items cut into pieces.  Slot = (tail item index) * k + piece (at most gridDim slots);
+// per slot and tile: m[128], l[128] and O[128][D], all fp32.
 struct PfScratch {
     float* ml;         // [slots][2 tiles][2][128]
     float* o;          // [slots][2 tiles][128][D]
@@ -328,6 +346,7 @@ struct PfScratch {
 template <int D>
 __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared& sh, const PfPlan& plan,
                                            const PfScratch& scr, const PfItem& it, int t, PfSoftmaxState& st) {
+    if (it.j1 <= it.j0) return true;  // an empty piece (more pieces than steps)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int j_end = min(it.j1, it.nkv[t]);
     if (j_end <= it.j0) return true;  // this tile has no step in this piece
@@ -432,7 +451,7 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
     tc_fence_after_sync();
     const bool row_ok = tok < p.C;
     __nv_bfloat16* dst = p.out + ((int64_t)tok * p.Hq + head) * D;
-    const bool whole = it.j0 == 0 && j_end == it.nkv[t];
+    const bool whole = it.j0 == 0 && j_end == it.nkv[t];  // this piece holds every step of the tile
     if (whole) {
         // epilogue of an item this CTA did alone: O / l -> bf16 -> out
         const float inv = 1.f / l_sum;
@@ -458,10 +477,12 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
     }
 
     // ---- the item is shared with other CTAs: publish this piece, the last piece to arrive merges all of them ----
-    const int cta = blockIdx.x;
-    const int first_cta = it.start / plan.spc;
-    const int last_cta = (it.start + it.nkv[t] - 1) / plan.spc;
-    const int my_slot = 2 * cta + (cta * plan.spc >= it.start ? 0 : 1);
+    // pieces of this item that hold steps of tile t: 0 .. last_piece (pieces are never empty: k <= nk / 4)
+    int last_piece = 0;
+    for (int i = 1; i < plan.pieces; ++i)
+        if (pf_piece_begin(it.nk, plan.pieces, i) < it.nkv[t]) last_piece = i;
+    const int n_mine = last_piece + 1;
+    const int my_slot = it.slot0 + it.piece;
     {
         float* ml = scr.ml + ((int64_t)my_slot * 2 + t) * 256;
         float* po = scr.o + (((int64_t)my_slot * 2 + t) * 128 + row) * D;
@@ -481,65 +502,76 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
     named_barrier_sync(2 + t, 128);
     if ((warp & 3) == 0 && lane == 0) scr.flags[t] = atomicAdd(&scr.tickets[it.item * 2 + t], 1);
     named_barrier_sync(2 + t, 128);
-    const bool merger = scr.flags[t] == last_cta - first_cta;
+    const bool merger = scr.flags[t] == n_mine - 1;
     named_barrier_sync(2 + t, 128);  // everyone has read the flag before a later piece may overwrite it
     if (!merger) return true;
     __threadfence();
     if ((warp & 3) == 0 && lane == 0) scr.tickets[it.item * 2 + t] = 0;  // re-armed for the next launch
+    const float* ml0 = scr.ml + ((int64_t)it.slot0 * 2 + t) * 256 + row;  // piece i: + i * 512 floats
     float m_all = -INFINITY;
-    for (int b = first_cta; b <= last_cta; ++b) {
-        const int slot = 2 * b + (b * plan.spc >= it.start ? 0 : 1);
-        m_all = fmaxf(m_all, __ldcg(scr.ml + ((int64_t)slot * 2 + t) * 256 + row));
-    }
-    float acc[D];
-#pragma unroll
-    for (int i = 0; i < D; ++i) acc[i] = 0.f;
+#pragma unroll 4
+    for (int i = 0; i <= last_piece; ++i) m_all = fmaxf(m_all, __ldcg(ml0 + (int64_t)i * 512));
+    // weights of the pieces: w_i = 2^(m_i - m_all); l = sum_i w_i l_i
     float l_all = 0.f;
-    for (int b = first_cta; b <= last_cta; ++b) {
-        const int slot = 2 * b + (b * plan.spc >= it.start ? 0 : 1);
-        const float* ml = scr.ml + ((int64_t)slot * 2 + t) * 256;
-        const float ms = __ldcg(ml + row);
-        const float w = ms == -INFINITY ? 0.f : fast_exp2(ms - m_all);
-        l_all += w * __ldcg(ml + 128 + row);
-        const float4* po = reinterpret_cast<const float4*>(scr.o + (((int64_t)slot * 2 + t) * 128 + row) * D);
+#pragma unroll 4
+    for (int i = 0; i <= last_piece; ++i) {
+        const float ms = __ldcg(ml0 + (int64_t)i * 512);
+        l_all += (ms == -INFINITY ? 0.f : fast_exp2(ms - m_all)) * __ldcg(ml0 + (int64_t)i * 512 + 128);
+    }
+    const float inv = 1.f / l_all;
+    // 64 output columns at a time keeps the accumulators small, so that the loads of two pieces are in flight
+    const float* o0 = scr.o + (((int64_t)it.slot0 * 2 + t) * 128 + row) * D;  // piece i: + i * 2 * 128 * D floats
+#pragma unroll 1
+    for (int c = 0; c < D / 64; ++c) {
+        float acc[64];
 #pragma unroll
-        for (int i = 0; i < D / 4; ++i) {
-            const float4 x = __ldcg(po + i);
-            acc[4 * i + 0] = fmaf(w, x.x, acc[4 * i + 0]);
-            acc[4 * i + 1] = fmaf(w, x.y, acc[4 * i + 1]);
-            acc[4 * i + 2] = fmaf(w, x.z, acc[4 * i + 2]);
-            acc[4 * i + 3] = fmaf(w, x.w, acc[4 * i + 3]);
+        for (int i = 0; i < 64; ++i) acc[i] = 0.f;
+#pragma unroll 2
+        for (int i = 0; i <= last_piece; ++i) {
+            const float ms = __ldcg(ml0 + (int64_t)i * 512);
+            const float w = ms == -INFINITY ? 0.f : fast_exp2(ms - m_all);
+            const float4* po = reinterpret_cast<const float4*>(o0 + (int64_t)i * 2 * 128 * D + c * 64);
+            float4 x[16];
+#pragma unroll
+            for (int q = 0; q < 16; ++q) x[q] = __ldcg(po + q);
+#pragma unroll
+            for (int q = 0; q < 16; ++q) {
+                acc[4 * q + 0] = fmaf(w, x[q].x, acc[4 * q + 0]);
+                acc[4 * q + 1] = fmaf(w, x[q].y, acc[4 * q + 1]);
+                acc[4 * q + 2] = fmaf(w, x[q].z, acc[4 * q + 2]);
+                acc[4 * q + 3] = fmaf(w, x[q].w, acc[4 * q + 3]);
+            }
+        }
+        if (row_ok) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                uint4 w;
+                w.x = pack_bf16x2(acc[8 * i + 0] * inv, acc[8 * i + 1] * inv);
+                w.y = pack_bf16x2(acc[8 * i + 2] * inv, acc[8 * i + 3] * inv);
+                w.z = pack_bf16x2(acc[8 * i + 4] * inv, acc[8 * i + 5] * inv);
+                w.w = pack_bf16x2(acc[8 * i + 6] * inv, acc[8 * i + 7] * inv);
+                *reinterpret_cast<uint4*>(dst + c * 64 + i * 8) = w;
+            }
         }
     }
-    if (row_ok) {
-        const float inv = 1.f / l_all;
-#pragma unroll
-        for (int i = 0; i < D / 8; ++i) {
-            uint4 w;
-            w.x = pack_bf16x2(acc[8 * i + 0] * inv, acc[8 * i + 1] * inv);
-            w.y = pack_bf16x2(acc[8 * i + 2] * inv, acc[8 * i + 3] * inv);
-            w.z = pack_bf16x2(acc[8 * i + 4] * inv, acc[8 * i + 5] * inv);
-            w.w = pack_bf16x2(acc[8 * i + 6] * inv, acc[8 * i + 7] * inv);
-            *reinterpret_cast<uint4*>(dst + i * 8) = w;
-        }
-        if (p.lse) p.lse[(int64_t)tok * p.Hq + head] = (m_all + __log2f(l_all)) * 0.6931471805599453f;
-    }
+    if (row_ok && p.lse) p.lse[(int64_t)tok * p.Hq + head] = (m_all + __log2f(l_all)) * 0.6931471805599453f;
     return true;
 }
 
 // ---- the prefill phase of one CTA ----------------------------------------------------------------------------------
+// `next` points at two shared-memory ints: the idle warp fetches the following entry from the global counter while
+// the current one is processed and leaves it in next[iteration parity]; everyone reads it after the piece barrier.
 template <int D>
 __device__ __forceinline__ void prefill_phase(const CUtensorMap* kv_map, const CUtensorMap* q_map, const MixedParams& p,
-                                              const PfShared& sh, const PfPlan& plan, const PfScratch& scr) {
+                                              const PfShared& sh, const PfPlan& plan, const PfScratch& scr, int first_entry,
+                                              volatile int* next) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int range_begin = min(plan.total_steps, (int)blockIdx.x * plan.spc);
-    const int range_end = min(plan.total_steps, range_begin + plan.spc);
     uint32_t prod_kv_it = 0, san_kv_it = 0;
     PfMmaState mma_state;
     PfSoftmaxState sm_state;
     // The softmax warpgroups hold a whole row of S in registers; the TMA / MMA / sanitizer warps need few.  The two
     // kinds of warps run separate loops (so that each gets its own register budget) and meet at a named barrier at
-    // the end of every piece.  (The caller guarantees a non-empty range: two register re-budgetings of a
+    // the end of every piece.  (The caller guarantees at least one entry: two register re-budgetings of a
     // warpgroup must be separated by a synchronisation of its warps.)
     auto piece_sync = [&]() {
         __syncwarp();
@@ -550,26 +582,30 @@ __device__ __forceinline__ void prefill_phase(const CUtensorMap* kv_map, const C
     };
     if (warp < 4) {
         setmaxnreg_dec<kPfRegsLight>();
-        for (int x = range_begin; x < range_end;) {
-            const PfItem it = pf_locate(p, plan, x, range_end);
+        int entry = first_entry;
+        for (int iter = 0; entry < plan.n_entries; ++iter) {
+            const PfItem it = pf_entry(p, plan, entry);
             if (warp == 0) {
-                if (lane == 0) pf_produce<D>(kv_map, q_map, p, sh, it, prod_kv_it);
+                if (lane == 0 && it.j1 > it.j0) pf_produce<D>(kv_map, q_map, p, sh, it, prod_kv_it);
             } else if (warp == 1) {
-                if (lane == 0) pf_mma<D>(p, sh, it, mma_state);
+                if (lane == 0 && it.j1 > it.j0) pf_mma<D>(p, sh, it, mma_state);
             } else if (warp == 2) {
-                pf_sanitize<D>(p, sh, it, san_kv_it);
+                if (it.j1 > it.j0) pf_sanitize<D>(p, sh, it, san_kv_it);
+            } else {
+                if (lane == 0) next[iter & 1] = atomicAdd(&p.ctrl[kCtrPrefill], 1);
             }
-            x = it.start + it.j1;
             if (!piece_sync()) break;
+            entry = next[iter & 1];
         }
         setmaxnreg_inc<kPfRegsLaunch>();
     } else {
         setmaxnreg_inc<kPfRegsHeavy>();
-        for (int x = range_begin; x < range_end;) {
-            const PfItem it = pf_locate(p, plan, x, range_end);
+        int entry = first_entry;
+        for (int iter = 0; entry < plan.n_entries; ++iter) {
+            const PfItem it = pf_entry(p, plan, entry);
             pf_softmax<D>(p, sh, plan, scr, it, (warp - 4) >> 2, sm_state);
-            x = it.start + it.j1;
             if (!piece_sync()) break;
+            entry = next[iter & 1];
         }
         setmaxnreg_dec<kPfRegsLaunch>();
     }
