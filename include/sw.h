@@ -117,6 +117,26 @@ sw_status sw_cost_probe(sw_ctx* ctx, void* const* kv_pools, int32_t layers, cons
                         void* out, int32_t warmup, int32_t reps, int64_t* p50_ns, int64_t* p99_ns,
                         int64_t* samples_ns, void* stream);
 
+/* (No counterpart in the paper.)  Decode-only attention for callers that cannot allocate device memory at all — for
+ * example a plugin or a real-time serving loop that runs inside someone else's memory pool, where cudaMalloc is
+ * forbidden or would synchronise the device, so neither a context nor a workspace can be created.  It computes what
+ * sw_mixed_attn_run computes for an iteration with chunk_len == 0 (q, out: device bf16 [n][num_q_heads][head_dim],
+ * lse: device fp32 [n][num_q_heads] or NULL; batch pointers are device pointers), but keeps its counters, tickets
+ * and split-KV partial results in a fixed array of SW_STATIC_SCRATCH_BYTES that is part of the library image: every
+ * GPU that loads the library holds that array until the process exits.  It calls no cudaMalloc / cudaFree and no
+ * allocating library routine.
+ * Limits: chunk_len must be 0, num_decode <= SW_STATIC_MAX_DECODE, num_kv_heads <= 8; anything larger is refused with
+ * SW_ERR_WORKSPACE (SW_ERR_UNSUPPORTED for a prefill chunk).
+ * The first call on a device looks up the array's device address, the device properties and the kernel attributes;
+ * make that first call outside any stream capture.  All calls share the one array: it is cleared where it must start
+ * at zero at the beginning of every call (on `stream`), so calls must not overlap on the GPU — issue them on one
+ * stream, or order them yourself; overlapping calls race on the scratch.  Not thread-safe for concurrent first calls.
+ * Asynchronous on `stream`; device-side problems are not reported by this variant (bad page ids are skipped). */
+#define SW_STATIC_MAX_DECODE 128
+#define SW_STATIC_SCRATCH_BYTES (7u * 1024u * 1024u)
+sw_status sw_decode_attn_static(const sw_layout* layout, int device, const void* kv_pool, const sw_batch* batch,
+                                const void* q, void* out, float* lse, void* stream);
+
 /* Wait for `stream` and read the device status words: *code is 0 or the first device-detected problem as an
  * sw_status (bad page id / length → SW_ERR_OUT_OF_RANGE, bounded wait expired → SW_ERR_DEVICE_TIMEOUT),
  * *detail an implementation-defined locator.  The words are cleared.  Returns *code as status. */

@@ -49,7 +49,8 @@ class sw_choice(C.Structure):
 
 EXPORTS = ["sw_workspace_bytes", "sw_create", "sw_destroy", "sw_kv_append", "sw_mixed_attn_run",
            "sw_mixed_iteration_host", "sw_cost_probe", "sw_check_status", "sw_cost_table_create",
-           "sw_cost_table_destroy", "sw_cost_table_lookup", "sw_choose_chunk", "sw_last_error"]
+           "sw_cost_table_destroy", "sw_cost_table_lookup", "sw_choose_chunk", "sw_last_error",
+           "sw_decode_attn_static"]
 
 _vp, _i32, _i64 = C.c_void_p, C.c_int32, C.c_int64
 _lib.sw_workspace_bytes.restype = C.c_size_t
@@ -62,6 +63,7 @@ _lib.sw_mixed_attn_run.argtypes = [_vp, _vp, C.POINTER(sw_batch), _vp, _vp, _vp,
 _lib.sw_mixed_iteration_host.argtypes = [_vp, _vp, C.POINTER(sw_batch), _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sw_cost_probe.argtypes = [_vp, C.POINTER(_vp), _i32, C.POINTER(sw_batch), _vp, _vp, _i32, _i32,
                                C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), _vp]
+_lib.sw_decode_attn_static.argtypes = [C.POINTER(sw_layout), C.c_int, _vp, C.POINTER(sw_batch), _vp, _vp, _vp, _vp]
 _lib.sw_check_status.argtypes = [_vp, _vp, C.POINTER(_i32), C.POINTER(_i32)]
 _lib.sw_cost_table_create.argtypes = [C.POINTER(_i32), _i32, C.POINTER(_i64), _i32, C.POINTER(_i32), _i32,
                                       C.POINTER(_i32), _i32, C.POINTER(_i64), C.c_int, C.c_int, C.POINTER(_vp)]
@@ -207,6 +209,16 @@ def sw_check_status(ctx: Context, stream=None, raise_on_error: bool = True):
     if st != SW_OK and raise_on_error:
         raise SwError(st, "sw_check_status")
     return int(code.value), int(detail.value)
+
+
+SW_STATIC_MAX_DECODE = 128
+
+
+def sw_decode_attn_static(layout: sw_layout, device: int, kv_pool, batch: DeviceBatch, q, out, lse=None, stream=None) -> None:
+    """Decode-only attention that allocates nothing: its scratch is a fixed array inside the library image, so it
+    needs neither a Context nor a workspace (for callers that may not call cudaMalloc)."""
+    _check(_lib.sw_decode_attn_static(C.byref(layout), device, _ptr(kv_pool), C.byref(batch.struct), _ptr(q), _ptr(out),
+                                      _ptr(lse), _stream_handle(stream)), "sw_decode_attn_static")
 
 
 def sw_debug_set_prefill_rows(ctx: Context, on: bool) -> None:
