@@ -14,7 +14,7 @@ constexpr int kMaxDecode = 2048;        // decode requests per iteration (prefix
 constexpr int kThreads = 384;           // 12 warps per CTA, one CTA per SM
 constexpr int kWarps = kThreads / 32;
 constexpr int kTargetItems = 4096;      // split-KV units aimed at per launch (bounds the partial-result scratch)
-constexpr int kMinSplitTokens = 256;    // never split a decode context finer than this
+constexpr int kMinSplitTokens = 128;    // never split a decode context finer than this
 constexpr int kMaxGroup = 8;            // query heads per KV head
 constexpr int kMaxCtas = 192;           // persistent CTAs (one per SM) the scratch is sized for
 constexpr int kMaxChunk = 65536;        // chunk tokens per iteration (256-row groups are planned in shared memory)

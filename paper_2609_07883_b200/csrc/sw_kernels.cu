@@ -151,8 +151,15 @@ __device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix
     }
     int total_pages = 0;
     block_exclusive_scan(pages_local, scratch, &total_pages);
-    const int per_head_target = max(1, p.target_items / p.Hkv);
-    int split_pages = (total_pages + per_head_target - 1) / per_head_target;
+    // Unit size.  Small batches are latency-bound: one round of units, as many as there are warps, gets every warp
+    // streaming at once.  Large batches are bandwidth-bound: a few rounds of smaller units shorten the tail.  Every
+    // request adds at most one ragged unit per head, hence the "- n".
+    const int per_head_warps = max(1, (int)gridDim.x * kWarps / p.Hkv);
+    const int one_round = (total_pages + per_head_warps - 1) / per_head_warps;  // pages per unit if run in one round
+    const int rounds = one_round <= 48 ? 1 : (one_round <= 160 ? 2 : 4);
+    int units_target = max(1, rounds * per_head_warps - p.n);
+    units_target = min(units_target, max(1, p.target_items / p.Hkv));
+    int split_pages = (total_pages + units_target - 1) / units_target;
     split_pages = max(split_pages, kMinSplitTokens / kPageSize);
     plan.split_tokens = split_pages * kPageSize;
     int units_local = 0;

@@ -1,0 +1,288 @@
+"""Iteration-level serving loop that drives the CUDA path with the SLOWeave controller (the bursty end-to-end workload).
+
+Each iteration decodes one token for every active request and optionally processes one prefill chunk of the oldest
+pending request (Sec. 4.1); requests that arrive during an iteration become eligible at its end.  The chunk is chosen
+by ``sw_choose_chunk`` (Algorithm 1) from the measured cost table; the iteration itself is KV append + the mixed
+attention launch over a stack of ``layers`` KV pools, and the virtual clock advances by its measured device time.
+Orchestration and bookkeeping only: chunk choice, append and attention all run in the library.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import sys
+import time
+from collections import deque
+from pathlib import Path
+
+import numpy as np
+
+from . import workloads as W
+
+MS = 1_000_000
+
+
+class PagePool:
+    """Free list of page ids (host side)."""
+
+    def __init__(self, num_pages: int, rng: np.random.Generator):
+        self.free = list(rng.permutation(num_pages).astype(np.int32))
+
+    def take(self, k: int):
+        if k > len(self.free):
+            return None
+        out = self.free[-k:] if k else []
+        del self.free[len(self.free) - k:]
+        return out
+
+    def give(self, ids):
+        self.free.extend(ids)
+
+
+class Request:
+    __slots__ = ("rid", "arrival", "prompt", "output", "prefilled", "generated", "pages", "last_token", "first_token",
+                 "gaps", "done_at")
+
+    def __init__(self, rid, arrival, prompt, output):
+        self.rid, self.arrival, self.prompt, self.output = rid, int(arrival), int(prompt), int(output)
+        self.prefilled = 0
+        self.generated = 0
+        self.pages = None
+        self.last_token = 0
+        self.first_token = None
+        self.gaps = []
+        self.done_at = None
+
+
+def gpu_executor(ctx, pools, shape: W.AttnShape, c_max: int, max_decode: int, seed: int = W.SEED_BASE + 44):
+    """Returns execute(batch) -> measured device nanoseconds of one iteration over the layer stack: per layer one
+    KV append and one mixed attention launch, timed with CUDA events on the current stream."""
+    import torch
+
+    from . import binding as B
+
+    dev = pools[0].device
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(seed)
+    rows_max = c_max + max_decode
+    q = torch.randn(rows_max, shape.num_q_heads, shape.head_dim, device=dev, generator=gen).to(torch.bfloat16)
+    k_new = torch.randn(rows_max, shape.num_kv_heads, shape.head_dim, device=dev, generator=gen).to(torch.bfloat16)
+    v_new = torch.randn(rows_max, shape.num_kv_heads, shape.head_dim, device=dev, generator=gen).to(torch.bfloat16)
+    out = torch.empty_like(q)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def execute(batch: W.MixedBatch) -> int:
+        db = B.DeviceBatch(batch, dev)
+        rows = batch.num_rows
+        ev0.record()
+        for pool_t in pools:
+            B.sw_kv_append(ctx, pool_t, db, k_new[:rows], v_new[:rows])
+            B.sw_mixed_attn_run(ctx, pool_t, db, q[:rows], out[:rows])
+        ev1.record()
+        ev1.synchronize()
+        return int(ev0.elapsed_time(ev1) * 1e6)
+
+    return execute
+
+
+def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, num_pages: int, policy: str = "sloweave",
+              c_max: int = 4096, margin_ppm: int = 50_000, margin_abs_ns: int = 0, quantum: int = 16, max_decode: int = 512,
+              ctx_cap: int | None = None, seed: int = W.SEED_BASE + 44, log=None) -> dict:
+    """Run the whole trace; returns statistics.  ``policy`` is "sloweave" or "fixed:<chunk>".  ``execute(batch)`` runs
+    one iteration and returns its duration in ns (``gpu_executor`` for the CUDA path).  ``ctx_cap`` clamps the total
+    context passed to the table lookup to the table's last grid point."""
+    from . import binding as B
+
+    S = shape.page_size
+    D_ns = int(tpot_ms * MS)
+    rng = np.random.default_rng(seed)
+    pool = PagePool(num_pages, rng)
+    reqs = [Request(i, trace["arrival_ns"][i], trace["prompt_len"][i], trace["output_len"][i])
+            for i in range(len(trace["arrival_ns"]))]
+    fixed_chunk = int(policy.split(":")[1]) if policy.startswith("fixed:") else None
+
+    pending, active = deque(), []
+    nxt, now, done = 0, 0, 0
+    iters = chunk_iters = 0
+    misses_chunk = misses_decode_only = infeasible_flags = stalled_for_memory = 0
+    chunks, iter_ns, pred_err = [], [], []
+    prefill_tokens = 0
+    wall0 = time.time()
+    while done < len(reqs):
+        while nxt < len(reqs) and reqs[nxt].arrival <= now:
+            pending.append(reqs[nxt])
+            nxt += 1
+        if not pending and not active:
+            now = reqs[nxt].arrival
+            continue
+        # ---- the controller's decision -----------------------------------------------------------------------
+        head = pending[0] if pending else None
+        if head is not None and head.pages is None:
+            need = -(-(head.prompt + head.output) // S)
+            head.pages = pool.take(need)           # blocks for the whole request are reserved when it is first scheduled
+            if head.pages is None:
+                stalled_for_memory += 1
+                head = None
+        n = len(active)
+        if n >= max_decode and head is not None:
+            head = None                             # the decode batch is full: no new request can finish its prefill
+        remaining = head.prompt - head.prefilled if head is not None else 0
+        deadlines = np.array([r.last_token + D_ns for r in active], dtype=np.int64)
+        total_ctx = sum(r.prompt + r.generated for r in active)
+        if ctx_cap is not None:
+            total_ctx = min(total_ctx, ctx_cap)
+        budget = int(deadlines.min() - now) if n else 0
+        predicted = 0
+        flags = 0
+        if fixed_chunk is not None:
+            c = min(fixed_chunk, remaining)
+        else:
+            q_eff = quantum if remaining >= quantum else 1   # the last few tokens of a prompt are below the quantum
+            ch = B.sw_choose_chunk(table if n else None, now, deadlines, total_ctx, head.prefilled if head else 0, remaining,
+                                   c_max=c_max, chunk_quantum=q_eff, margin_abs_ns=margin_abs_ns, margin_ppm=margin_ppm)
+            c, flags, predicted = ch.chunk, ch.flags, ch.predicted_ns
+        if n == 0 and c == 0:
+            # nothing to run (memory stall with an idle GPU): wait for the next arrival or fail loudly
+            if nxt < len(reqs):
+                now = max(now, reqs[nxt].arrival)
+                continue
+            raise RuntimeError("serving loop stalled: pool too small for the remaining requests")
+        # ---- build the iteration and run it over the layer stack -----------------------------------------------
+        P = head.prefilled if (head is not None and c > 0) else 0
+        lens = np.array([r.prompt + r.generated for r in active], dtype=np.int32)
+        per = [(-(-int(L) // S)) for L in lens]
+        indptr = np.zeros(n + 1, dtype=np.int32)
+        indptr[1:] = np.cumsum(per)
+        dpages = np.concatenate([np.asarray(r.pages[:k], dtype=np.int32) for r, k in zip(active, per)]) if n else \
+            np.zeros(0, np.int32)
+        ppages = np.asarray(head.pages[: -(-(P + c) // S)], dtype=np.int32) if c > 0 else np.zeros(0, np.int32)
+        batch = W.MixedBatch(shape, num_pages, P, c, ppages, lens, indptr, dpages)
+        dt = int(execute(batch))
+        now += dt
+        iters += 1
+        iter_ns.append(dt)
+        # ---- bookkeeping ------------------------------------------------------------------------------------------
+        if n and dt > budget:
+            if c > 0:
+                misses_chunk += 1
+            else:
+                misses_decode_only += 1
+        if flags & B.SW_F_DECODE_INFEASIBLE:
+            infeasible_flags += 1
+        if predicted and n:
+            pred_err.append(dt - predicted)
+        still = []
+        for r in active:
+            r.generated += 1
+            r.gaps.append(now - r.last_token)
+            r.last_token = now
+            if r.generated >= r.output:
+                r.done_at = now
+                pool.give(r.pages)
+                r.pages = None
+                done += 1
+            else:
+                still.append(r)
+        active = still
+        if c > 0:
+            chunk_iters += 1
+            chunks.append(c)
+            prefill_tokens += c
+            head.prefilled += c
+            if head.prefilled >= head.prompt:      # the iteration that finishes the prompt emits the first token
+                pending.popleft()
+                head.first_token = now
+                head.last_token = now
+                head.generated = 1
+                if head.output <= 1:
+                    head.done_at = now
+                    pool.give(head.pages)
+                    head.pages = None
+                    done += 1
+                else:
+                    active.append(head)
+        if log and iters % 2000 == 0:
+            log(f"  iter {iters}: t={now / 1e9:.2f}s done={done} active={len(active)} pending={len(pending)} "
+                f"wall={time.time() - wall0:.0f}s")
+    ttft = np.array([r.first_token - r.arrival for r in reqs], dtype=np.float64) / MS
+    p99_gap = np.array([np.percentile(r.gaps, 99) if r.gaps else 0.0 for r in reqs]) / MS
+    duration_s = now / 1e9
+    return {
+        "policy": policy, "tpot_ms": tpot_ms, "requests": len(reqs), "iterations": iters, "chunk_iterations": chunk_iters,
+        "deadline_misses_with_chunk": misses_chunk, "deadline_misses_decode_only": misses_decode_only,
+        "decode_infeasible_flags": infeasible_flags, "memory_stalls": stalled_for_memory,
+        "trace_duration_s": duration_s, "prefill_tokens": prefill_tokens,
+        "prefill_tokens_per_s": prefill_tokens / duration_s, "decode_tokens_per_s": float(sum(r.output for r in reqs)) / duration_s,
+        "mean_chunk": float(np.mean(chunks)) if chunks else 0.0, "p99_chunk": float(np.percentile(chunks, 99)) if chunks else 0.0,
+        "iter_ms_p50": float(np.percentile(iter_ns, 50)) / MS, "iter_ms_p99": float(np.percentile(iter_ns, 99)) / MS,
+        "ttft_ms_p50": float(np.percentile(ttft, 50)), "ttft_ms_p99": float(np.percentile(ttft, 99)),
+        "tpot_ms_p99_of_request_p99": float(np.percentile(p99_gap, 99)),
+        "requests_meeting_tpot": int(np.sum(p99_gap <= tpot_ms)),
+        "prediction_error_ms_p99": float(np.percentile(pred_err, 99)) / MS if pred_err else 0.0,
+        "margin_ppm": margin_ppm, "c_max": c_max, "quantum": quantum, "wall_s": time.time() - wall0,
+    }
+
+
+def main(argv=None):
+    import torch
+
+    from . import binding as B
+    from . import build, profiler
+
+    ap = argparse.ArgumentParser(description="bursty serving loop over a layer stack with the SLOWeave controller")
+    ap.add_argument("--requests", type=int, default=2000)
+    ap.add_argument("--layers", type=int, default=32)
+    ap.add_argument("--pages", type=int, default=40960, help="pages per layer pool")
+    ap.add_argument("--tpot-ms", type=float, nargs="+", default=[10.0, 25.0])
+    ap.add_argument("--policies", nargs="+", default=["sloweave"])
+    ap.add_argument("--c-max", type=int, default=4096)
+    ap.add_argument("--margin-ppm", type=int, default=50_000)
+    ap.add_argument("--table", default=None, help="JSON cost table to reuse; measured first when absent")
+    ap.add_argument("--table-reps", type=int, default=8)
+    ap.add_argument("--out", default="gpurun_out/bursty.json")
+    args = ap.parse_args(argv)
+
+    build.build()
+    dev = torch.device("cuda", 0)
+    shape = W.LLAMA
+    max_decode = 512
+    ctx = B.Context(shape, args.pages, args.c_max, max_decode, args.pages + 64)
+    pools = []
+    for layer in range(args.layers):
+        t = torch.empty(args.pages * shape.page_elems, dtype=torch.bfloat16, device=dev)
+        W.fill_normal_bf16_(t, W.SEED_BASE + 400 + layer)
+        pools.append(t)
+    log = lambda s: print(s, file=sys.stderr, flush=True)
+    if args.table and Path(args.table).exists():
+        tab = profiler.load_table(args.table)
+    else:
+        tokens = args.pages * shape.page_size
+        n_grid = [1, 4, 16, 48, 128, 256, 512]
+        ctx_grid = [t for t in (8192, 65536, 196608, 393216) if t < tokens - 40000] + [tokens - 40000]
+        prefix_grid = [0, 2048, 8192, 32768]
+        chunk_grid = [0, 16, 64, 128, 256, 512, 1024, 2048, 4096]
+        log(f"measuring cost table: {len(n_grid) * len(ctx_grid) * len(prefix_grid) * len(chunk_grid)} points, {args.layers} layers")
+        tab = profiler.measure_table(ctx, pools, shape, args.pages, n_grid, ctx_grid, prefix_grid, chunk_grid,
+                                     reps=args.table_reps, warmup=2, progress=log)
+        if args.table:
+            profiler.save_table(tab, args.table)
+    table = profiler.to_cost_table(tab)
+    trace = W.bursty_trace(num_requests=args.requests)
+    execute = gpu_executor(ctx, pools, shape, args.c_max, max_decode)
+    results = {"layers": args.layers, "pages_per_layer": args.pages, "table_points": int(np.prod(np.shape(tab["p99_ns"]))),
+               "runs": []}
+    for tpot in args.tpot_ms:
+        for policy in args.policies:
+            log(f"run: tpot={tpot} ms policy={policy}")
+            res = run_trace(trace, tpot, table, execute, shape, args.pages, policy=policy, c_max=args.c_max,
+                            margin_ppm=args.margin_ppm, max_decode=max_decode, ctx_cap=tab["ctx_grid"][-1], log=log)
+            B.sw_check_status(ctx)
+            log(json.dumps(res))
+            results["runs"].append(res)
+    Path(args.out).parent.mkdir(parents=True, exist_ok=True)
+    Path(args.out).write_text(json.dumps(results, indent=1))
+    print(json.dumps(results))
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,69 @@
+"""The iteration-level serving loop on CPU: the controller is the library's (host-only), the executor is the analytic
+cost model of Sec. 4.1, so the loop's scheduling semantics and Proposition 1 can be checked without a GPU."""
+import numpy as np
+import pytest
+
+from paper_2609_07883_b200 import workloads as W
+
+MS = 1_000_000
+
+
+@pytest.fixture(scope="module")
+def env(oracle):
+    from paper_2609_07883_b200 import build
+
+    build.build()
+    from paper_2609_07883_b200 import binding as B
+    from paper_2609_07883_b200 import serving
+
+    n_values = list(range(1, 97))
+    chunk_grid = list(range(0, 2049))
+    cost = np.array([[oracle.analytic_cost_ns(n, c) for c in chunk_grid] for n in n_values], dtype=np.int64)
+    table = B.CostTable(n_values, [1 << 40], [1 << 30], chunk_grid, cost.reshape(len(n_values), 1, 1, -1))
+
+    def execute(batch):
+        return oracle.analytic_cost_ns(batch.num_decode, batch.chunk_len)
+
+    trace = W.bursty_trace(num_requests=120, rate_low=20.0, rate_high=80.0, mean_dwell_s=1.0, prompt_median=600.0,
+                           prompt_clip=(32, 4096), mean_output=40.0, rng=np.random.default_rng(5))
+    return B, serving, table, execute, trace
+
+
+def test_sloweave_meets_every_deadline_under_an_exact_monotone_cost(env):
+    B, serving, table, execute, trace = env
+    res = serving.run_trace(trace, 25.0, table, execute, W.LLAMA, 8192, policy="sloweave", c_max=2048, margin_ppm=0,
+                            quantum=16, max_decode=96)
+    assert res["deadline_misses_with_chunk"] == 0            # Proposition 1 (i)
+    assert res["deadline_misses_decode_only"] == res["decode_infeasible_flags"] == 0   # n <= 96 decodes fit 25 ms
+    assert res["prefill_tokens"] == int(trace["prompt_len"].sum())
+    assert res["requests_meeting_tpot"] == 120
+    assert res["tpot_ms_p99_of_request_p99"] <= 25.0
+    assert res["chunk_iterations"] > 0 and res["mean_chunk"] > 16
+
+
+def test_a_large_fixed_chunk_misses_deadlines_that_sloweave_meets(env):
+    B, serving, table, execute, trace = env
+    fixed = serving.run_trace(trace, 10.0, table, execute, W.LLAMA, 8192, policy="fixed:2048", c_max=2048, max_decode=96)
+    adaptive = serving.run_trace(trace, 10.0, table, execute, W.LLAMA, 8192, policy="sloweave", c_max=2048, margin_ppm=0,
+                                 max_decode=96)
+    assert fixed["deadline_misses_with_chunk"] > 0
+    assert adaptive["deadline_misses_with_chunk"] == 0
+    assert adaptive["prefill_tokens"] == fixed["prefill_tokens"] == int(trace["prompt_len"].sum())
+
+
+def test_arrivals_become_eligible_at_iteration_end_and_tokens_add_up(env):
+    B, serving, table, execute, trace = env
+    seen = []
+
+    def spy(batch):
+        seen.append((batch.num_decode, batch.chunk_len, int(batch.total_decode_ctx)))
+        return execute(batch)
+
+    res = serving.run_trace(trace, 25.0, table, spy, W.LLAMA, 8192, policy="sloweave", c_max=2048, margin_ppm=0,
+                            max_decode=96)
+    assert len(seen) == res["iterations"]
+    # every iteration decodes one token per active request: decode tokens = sum(output) - one first token per request
+    # (the first token comes out of the iteration that finishes the prompt)
+    assert sum(n for n, _, _ in seen) == int(trace["output_len"].sum()) - int((trace["output_len"] >= 1).sum())
+    assert sum(c for _, c, _ in seen) == int(trace["prompt_len"].sum())
+    assert res["ttft_ms_p50"] > 0 and res["trace_duration_s"] * 1e9 >= trace["arrival_ns"][-1]
