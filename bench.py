@@ -170,12 +170,38 @@ def host_tensors_for(batch: W.MixedBatch, seed: int) -> dict:
 
 
 # ---------------------------------------------------------------------------------------------------------------
+# multi-process plumbing (one process per GPU; replicas only: the path has no exchange step)
+# ---------------------------------------------------------------------------------------------------------------
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def reduce_max_over_ranks(x: float, device=None) -> float:
+    """max over ranks of a per-rank duration (identity when no process group is initialised)."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_result(per_rank_us: float, world: int, chunk: int, decodes: int, device=None) -> dict:
+    """Whole-job numbers of N independent replicas: the iteration time is the slowest rank's, throughputs add up."""
+    us = reduce_max_over_ranks(per_rank_us, device)
+    return {"value": us, "iterations_per_s": world / (us * 1e-6), "prefill_tokens_per_s": world * chunk / (us * 1e-6),
+            "decode_tokens_per_s": world * decodes / (us * 1e-6)}
+
+
+# ---------------------------------------------------------------------------------------------------------------
 # main legs
 # ---------------------------------------------------------------------------------------------------------------
 def run_reference(args) -> dict:
-    rank = int(os.environ.get("RANK", "0"))
+    rank, _, _ = dist_env()
     if rank != 0:
-        return {}
+        return {}          # under torchrun only rank 0 runs the oracle; the others exit 0 without work
     batch = make_workload(args, 0)
     tensors = host_tensors_for(batch, 1234)
     times = []
@@ -211,9 +237,7 @@ def run_ours(args) -> dict:
 
     from paper_2609_07883_b200 import build
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank, local_rank, world = dist_env()
     if rank == 0:
         build.build()
     if world > 1:
@@ -254,11 +278,7 @@ def run_ours(args) -> dict:
             torch.cuda.synchronize()
 
     def reduce_max(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return reduce_max_over_ranks(x, dev)
 
     for i in range(args.warmup):
         step(i)
@@ -276,7 +296,9 @@ def run_ours(args) -> dict:
         step(i)
     e1.record()
     sync_all()
-    ms_total = reduce_max(e0.elapsed_time(e1))
+    ms_local = e0.elapsed_time(e1)
+    agg = aggregate_result(ms_local / args.steps * 1e3, world, batch.chunk_len, batch.num_decode, dev)
+    ms_total = agg["value"] * args.steps / 1e3
     # (2) the attention launch alone (dominant kernel) for the roofline, same stream, same rotation
     a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a0.record()
@@ -316,9 +338,9 @@ def run_ours(args) -> dict:
         "metric": "mixed_iteration_us", "value": us, "unit": "us", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(args, batch),
-        "iterations_per_s": world / (us * 1e-6),
-        "prefill_tokens_per_s": world * batch.chunk_len / (us * 1e-6),
-        "decode_tokens_per_s": world * batch.num_decode / (us * 1e-6),
+        "iterations_per_s": agg["iterations_per_s"],
+        "prefill_tokens_per_s": agg["prefill_tokens_per_s"],
+        "decode_tokens_per_s": agg["decode_tokens_per_s"],
         "attn_launch_us": attn_ms * 1e3,
         "roofline": {"bound": "hbm", "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved_gbs / peaks["hbm_gbs"], "traffic": None, "peak_kind": f"of {peak_kind}",

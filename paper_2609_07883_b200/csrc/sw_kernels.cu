@@ -148,6 +148,8 @@ __device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix
     for (int i = beg; i < end; ++i) {
         const int len = p.decode_kv_len[i];
         pages_local += len > 0 ? (len + kPageSize - 1) / kPageSize : 0;
+        // the units read these offsets later: bring their lines into L1 now
+        asm volatile("prefetch.global.L1 [%0];" ::"l"(p.decode_page_indptr + i));
     }
     int total_pages = 0;
     block_exclusive_scan(pages_local, scratch, &total_pages);
@@ -413,12 +415,14 @@ __device__ bool run_unit(const CUtensorMap* kv_map, const MixedParams& p, const 
     const int slot0 = u.slot - u.split * p.Hkv;
     for (int r = 0; r < g; ++r) {
         float m_all = -INFINITY;
+#pragma unroll 4
         for (int sidx = 0; sidx < u.nsplit; ++sidx)
             m_all = fmaxf(m_all, __ldcg(&p.part_ml[(int64_t)(slot0 + sidx * p.Hkv) * (2 * kMaxGroup) + r]));
         float l_all = 0.f;
         float acc[D / 32];
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) acc[c] = 0.f;
+#pragma unroll 4
         for (int sidx = 0; sidx < u.nsplit; ++sidx) {
             const int64_t sl = slot0 + sidx * p.Hkv;
             const float ms = __ldcg(&p.part_ml[sl * (2 * kMaxGroup) + r]);
@@ -514,10 +518,18 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
         ring.buf = base + warp * kStages * Geo<D>::kStageBytes;
         ring.bar = base + Geo<D>::kBarOffset + warp * kStages * 8;
         ring.it = 0;
+        // first unit by warp index (no round trip to the counter), the following ones from the shared counter
+        const int total_warps = (int)gridDim.x * kWarps;
+        bool first = true;
         while (true) {
             int item = 0;
-            if (lane == 0) item = atomicAdd(&p.ctrl[kCtrWork], 1);
-            item = __shfl_sync(0xffffffffu, item, 0);
+            if (first) {
+                item = (int)blockIdx.x * kWarps + warp;
+                first = false;
+            } else {
+                if (lane == 0) item = total_warps + atomicAdd(&p.ctrl[kCtrWork], 1);
+                item = __shfl_sync(0xffffffffu, item, 0);
+            }
             if (item >= plan.total_items) break;
             Unit u;
             bool ok = true;

@@ -286,7 +286,7 @@ __device__ __forceinline__ bool pf_mma(const MixedParams& p, const PfShared& sh,
         const uint32_t s = cur & 1, n = cur >> 1;
         if (!pf_wait(sh, kBarVFull + s, n & 1, p.ctrl, 6)) return false;
         const bool more = j + 1 < it.j1;
-        if (more && !pf_wait(sh, kBarKFull + (s ^ 1), ((cur + 1) >> 1) & 1, p.ctrl, 7)) return false;
+        bool k_ready = false;  // K of tile j+1 is awaited as late as possible: right before its first use
         for (int t = 0; t < 2; ++t) {
             if (act(t, j)) {
                 if (!pf_wait(sh, kBarPFull + t, st.p_cnt[t] & 1, p.ctrl, 8)) return false;
@@ -295,7 +295,13 @@ __device__ __forceinline__ bool pf_mma(const MixedParams& p, const PfShared& sh,
                 pf_issue_pv<D>(sh, t, s, j == it.j0);
             }
             if (t == last_active(j)) tc_commit(sh.bars + (kBarVEmpty + s) * 8);
-            if (act(t, j + 1)) pf_issue_qk<D>(sh, t, s ^ 1);
+            if (act(t, j + 1)) {
+                if (!k_ready) {
+                    if (!pf_wait(sh, kBarKFull + (s ^ 1), ((cur + 1) >> 1) & 1, p.ctrl, 7)) return false;
+                    k_ready = true;
+                }
+                pf_issue_qk<D>(sh, t, s ^ 1);
+            }
             if (more && t == last_active(j + 1)) tc_commit(sh.bars + (kBarKEmpty + (s ^ 1)) * 8);
         }
     }

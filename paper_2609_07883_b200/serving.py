@@ -235,6 +235,8 @@ def main(argv=None):
     ap.add_argument("--pages", type=int, default=40960, help="pages per layer pool")
     ap.add_argument("--tpot-ms", type=float, nargs="+", default=[10.0, 25.0])
     ap.add_argument("--policies", nargs="+", default=["sloweave"])
+    ap.add_argument("--rate-scale", type=float, nargs="+", default=[1.0],
+                    help="divide the trace's arrival times by this factor (1 = the stated 2 / 20 req/s)")
     ap.add_argument("--c-max", type=int, default=4096)
     ap.add_argument("--margin-ppm", type=int, default=50_000)
     ap.add_argument("--table", default=None, help="JSON cost table to reuse; measured first when absent")
@@ -258,9 +260,11 @@ def main(argv=None):
     else:
         tokens = args.pages * shape.page_size
         n_grid = [1, 4, 16, 48, 128, 256, 512]
-        ctx_grid = [t for t in (8192, 65536, 196608, 393216) if t < tokens - 40000] + [tokens - 40000]
         prefix_grid = [0, 2048, 8192, 32768]
         chunk_grid = [0, 16, 64, 128, 256, 512, 1024, 2048, 4096]
+        # the largest context that still leaves room for the longest prompt piece and one ragged page per request
+        ctx_top = tokens - (prefix_grid[-1] + chunk_grid[-1]) - shape.page_size * (n_grid[-1] + 64)
+        ctx_grid = [t for t in (8192, 65536, 196608, 393216) if t < ctx_top] + [ctx_top]
         log(f"measuring cost table: {len(n_grid) * len(ctx_grid) * len(prefix_grid) * len(chunk_grid)} points, {args.layers} layers")
         tab = profiler.measure_table(ctx, pools, shape, args.pages, n_grid, ctx_grid, prefix_grid, chunk_grid,
                                      reps=args.table_reps, warmup=2, progress=log)
@@ -271,14 +275,17 @@ def main(argv=None):
     execute = gpu_executor(ctx, pools, shape, args.c_max, max_decode)
     results = {"layers": args.layers, "pages_per_layer": args.pages, "table_points": int(np.prod(np.shape(tab["p99_ns"]))),
                "runs": []}
-    for tpot in args.tpot_ms:
-        for policy in args.policies:
-            log(f"run: tpot={tpot} ms policy={policy}")
-            res = run_trace(trace, tpot, table, execute, shape, args.pages, policy=policy, c_max=args.c_max,
-                            margin_ppm=args.margin_ppm, max_decode=max_decode, ctx_cap=tab["ctx_grid"][-1], log=log)
-            B.sw_check_status(ctx)
-            log(json.dumps(res))
-            results["runs"].append(res)
+    for scale in args.rate_scale:
+        scaled = dict(trace, arrival_ns=(trace["arrival_ns"] / scale).astype(np.int64))
+        for tpot in args.tpot_ms:
+            for policy in args.policies:
+                log(f"run: rate x{scale} tpot={tpot} ms policy={policy}")
+                res = run_trace(scaled, tpot, table, execute, shape, args.pages, policy=policy, c_max=args.c_max,
+                                margin_ppm=args.margin_ppm, max_decode=max_decode, ctx_cap=tab["ctx_grid"][-1], log=log)
+                B.sw_check_status(ctx)
+                res["rate_scale"] = scale
+                log(json.dumps(res))
+                results["runs"].append(res)
     Path(args.out).parent.mkdir(parents=True, exist_ok=True)
     Path(args.out).write_text(json.dumps(results, indent=1))
     print(json.dumps(results))

@@ -1,0 +1,135 @@
+"""Full-size parity: the workloads bench.py times (and the larger ones), in the same launch configuration, checked on
+sampled outputs that the oracle computes one by one; the KV pools after append are compared whole, bit for bit."""
+import numpy as np
+import pytest
+
+from paper_2609_07883_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import torch
+
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_07883_b200 import build
+
+    build.build()
+    from tests import gpu_util
+
+    return gpu_util
+
+
+def run_case(gpu, oracle, batch, pairs, seed, what):
+    import torch
+
+    from paper_2609_07883_b200 import binding as B
+
+    dev = torch.device("cuda", 0)
+    sh = batch.shape
+    total_pages = int(batch.prefill_pages.shape[0] + batch.decode_pages.shape[0])
+    ctx = B.Context(sh, batch.num_pages, max(batch.chunk_len, 1), max(batch.num_decode, 1), total_pages + 16)
+    db = B.DeviceBatch(batch, dev)
+    pool = torch.empty(batch.num_pages * sh.page_elems, dtype=torch.bfloat16, device=dev)
+    W.fill_normal_bf16_(pool, seed)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(seed + 1)
+    R = batch.num_rows
+    q = torch.randn(R, sh.num_q_heads, sh.head_dim, device=dev, generator=gen).to(torch.bfloat16)
+    k_new = torch.randn(R, sh.num_kv_heads, sh.head_dim, device=dev, generator=gen).to(torch.bfloat16)
+    v_new = torch.randn(R, sh.num_kv_heads, sh.head_dim, device=dev, generator=gen).to(torch.bfloat16)
+    out = torch.zeros_like(q)
+    lse = torch.zeros(R, sh.num_q_heads, dtype=torch.float32, device=dev)
+    host_pool = gpu.torch_to_bits(pool)          # the inputs, before the append
+    B.sw_kv_append(ctx, pool, db, k_new, v_new)
+    B.sw_mixed_attn_run(ctx, pool, db, q, out, lse)
+    torch.cuda.synchronize()
+    assert B.sw_check_status(ctx, raise_on_error=False) == (0, 0)
+    assert oracle.kv_append(host_pool, batch, gpu.torch_to_bits(k_new), gpu.torch_to_bits(v_new)) == 0
+    assert np.array_equal(gpu.torch_to_bits(pool), host_pool), f"{what}: pool differs after append"
+    pairs = np.asarray(pairs, dtype=np.int32)
+    ref, ref_lse, _ = oracle.mixed_attention(host_pool, batch, gpu.torch_to_bits(q), pairs=pairs)
+    got = W.bf16_bits_to_f64(gpu.torch_to_bits(out))[pairs[:, 0], pairs[:, 1]]
+    got_lse = lse.cpu().numpy().astype(np.float64)[pairs[:, 0], pairs[:, 1]]
+    return gpu.compare(got, got_lse, ref, ref_lse, what)
+
+
+def sample_pairs(batch, rng, chunk_rows, n_decode_extra):
+    C, n, Hq = batch.chunk_len, batch.num_decode, batch.shape.num_q_heads
+    rows = [r for r in chunk_rows if 0 <= r < C]
+    if n:
+        lens = batch.decode_kv_len
+        rows += [C + int(np.argmin(lens)), C + int(np.argmax(lens))]
+        rows += [C + int(i) for i in rng.choice(n, size=min(n, n_decode_extra), replace=False)]
+    return [(r, int(rng.integers(0, Hq))) for r in rows]
+
+
+def test_chat_workload_as_benchmarked(gpu, oracle):
+    rng = W.rng_for(1)
+    batch = W.chat_batch(n=64, chunk_len=512, prefix_len=512, rng=rng)
+    pairs = sample_pairs(batch, np.random.default_rng(1), [0, 1, 15, 16, 31, 32, 63, 64, 127, 128, 255, 256, 383, 511], 12)
+    run_case(gpu, oracle, batch, pairs, 101, "chat n=64 C=512 P=512")
+
+
+def test_mixed_workload_cost_surface_point(gpu, oracle):
+    rng = W.rng_for(2)
+    batch = W.mixed_batch(1024, 4096, n=128, rng=rng)
+    pairs = sample_pairs(batch, np.random.default_rng(2), [0, 31, 32, 127, 128, 129, 511, 512, 1000, 1023], 16)
+    run_case(gpu, oracle, batch, pairs, 102, "mixed n=128 C=1024 P=4096")
+
+
+def test_long_context_workload(gpu, oracle):
+    rng = W.rng_for(3)
+    batch = W.long_batch(1024, 98304, n=16, rng=rng)
+    pairs = sample_pairs(batch, np.random.default_rng(3), [0, 1, 63, 64, 512, 1023], 6)
+    run_case(gpu, oracle, batch, pairs, 103, "long n=16 C=1024 P=98304")
+
+
+def test_page_ids_above_two_to_the_twenty(gpu, oracle):
+    """A 70 GB pool (1.1 M pages of 64 KB) with the live pages scattered over all of it: byte offsets pass 2^36."""
+    import torch
+
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    num_pages = (1 << 20) + 4096
+    if free < num_pages * W.LLAMA.page_elems * 2 + (8 << 30):
+        pytest.skip("not enough free device memory for the large pool")
+    rng = np.random.default_rng(9)
+    batch = W.make_batch(W.LLAMA, num_pages, [3000, 17, 700], 1000, 200, rng)
+    assert int(max(batch.decode_pages.max(), batch.prefill_pages.max())) > (1 << 19)
+    from paper_2609_07883_b200 import binding as B
+
+    dev = torch.device("cuda", 0)
+    sh = batch.shape
+    ctx = B.Context(sh, num_pages, 200, 3, 512)
+    db = B.DeviceBatch(batch, dev)
+    pool = torch.zeros(num_pages * sh.page_elems, dtype=torch.bfloat16, device=dev)
+    # fill only the live pages with data; the oracle works on a compact copy with renumbered pages
+    live = np.concatenate([batch.decode_pages, batch.prefill_pages]).astype(np.int64)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(77)
+    data = torch.randn(len(live), sh.page_elems, device=dev, generator=gen).to(torch.bfloat16)
+    pool.view(num_pages, sh.page_elems)[torch.from_numpy(live).to(dev)] = data
+    R = batch.num_rows
+    q = torch.randn(R, sh.num_q_heads, sh.head_dim, device=dev, generator=gen).to(torch.bfloat16)
+    k_new = torch.randn(R, sh.num_kv_heads, sh.head_dim, device=dev, generator=gen).to(torch.bfloat16)
+    v_new = torch.randn(R, sh.num_kv_heads, sh.head_dim, device=dev, generator=gen).to(torch.bfloat16)
+    out = torch.zeros_like(q)
+    B.sw_kv_append(ctx, pool, db, k_new, v_new)
+    B.sw_mixed_attn_run(ctx, pool, db, q, out)
+    torch.cuda.synchronize()
+    assert B.sw_check_status(ctx, raise_on_error=False) == (0, 0)
+    compact = W.MixedBatch(sh, len(live), batch.prefix_len, batch.chunk_len,
+                           np.arange(len(batch.decode_pages), len(live), dtype=np.int32), batch.decode_kv_len,
+                           batch.decode_page_indptr, np.arange(len(batch.decode_pages), dtype=np.int32))
+    host_pool = gpu.torch_to_bits(data).reshape(-1).copy()
+    assert oracle.kv_append(host_pool, compact, gpu.torch_to_bits(k_new), gpu.torch_to_bits(v_new)) == 0
+    got_pages = gpu.torch_to_bits(pool.view(num_pages, sh.page_elems)[torch.from_numpy(live).to(dev)])
+    assert np.array_equal(got_pages.reshape(-1), host_pool)            # append landed in the right far-away pages
+    others = np.setdiff1d(rng.integers(0, num_pages, size=4096), live)                 # and nowhere else (sampled)
+    untouched = pool.view(num_pages, sh.page_elems)[torch.from_numpy(others).to(dev)].view(torch.int16)
+    assert int(torch.count_nonzero(untouched).item()) == 0
+    ref, _, _ = oracle.mixed_attention(host_pool, compact, gpu.torch_to_bits(q))
+    gpu.compare(W.bf16_bits_to_f64(gpu.torch_to_bits(out)).reshape(-1, sh.head_dim), None, ref, None, "far pages")
