@@ -518,18 +518,10 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
         ring.buf = base + warp * kStages * Geo<D>::kStageBytes;
         ring.bar = base + Geo<D>::kBarOffset + warp * kStages * 8;
         ring.it = 0;
-        // first unit by warp index (no round trip to the counter), the following ones from the shared counter
-        const int total_warps = (int)gridDim.x * kWarps;
-        bool first = true;
         while (true) {
             int item = 0;
-            if (first) {
-                item = (int)blockIdx.x * kWarps + warp;
-                first = false;
-            } else {
-                if (lane == 0) item = total_warps + atomicAdd(&p.ctrl[kCtrWork], 1);
-                item = __shfl_sync(0xffffffffu, item, 0);
-            }
+            if (lane == 0) item = atomicAdd(&p.ctrl[kCtrWork], 1);
+            item = __shfl_sync(0xffffffffu, item, 0);
             if (item >= plan.total_items) break;
             Unit u;
             bool ok = true;
@@ -560,8 +552,11 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
                 u.len = p.decode_kv_len[i];
                 u.split = unit - unit_prefix[i];
                 u.nsplit = unit_prefix[i + 1] - unit_prefix[i];
-                u.t_begin = u.split * plan.split_tokens;
-                u.t_end = min(u.len, u.t_begin + plan.split_tokens);
+                // the request's pages are shared out evenly among its units (no ragged last unit)
+                const int req_pages = (u.len + kPageSize - 1) / kPageSize;
+                const int unit_pages = (req_pages + u.nsplit - 1) / u.nsplit;
+                u.t_begin = min(u.len, u.split * unit_pages * kPageSize);
+                u.t_end = min(u.len, u.t_begin + unit_pages * kPageSize);
                 u.ticket = i * p.Hkv + u.kvh;
                 u.slot = di;
                 const int beg = p.decode_page_indptr[i];
