@@ -27,6 +27,10 @@ __device__ __forceinline__ void report(int32_t* ctrl, int code, int site, int in
 // ---------------------------------------------------------------------------------------------------------------
 // One thread per (row, 16-byte piece of the row's Hkv*D elements); it copies that piece of K and of V.
 __global__ void sw_kv_append_kernel(const AppendParams p) {
+    // launched with programmatic stream serialization: it may start while the previous kernel (the attention of
+    // the previous iteration, possibly still reading this pool) drains; nothing is touched before this wait
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int pieces_per_row = p.Hkv * p.D / 8;
     const int64_t total = (int64_t)(p.C + p.n) * pieces_per_row;
     for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
@@ -79,8 +83,17 @@ cudaError_t launch_kv_append(const AppendParams& p, cudaStream_t stream) {
     const int threads = 256;
     int64_t blocks = (total + threads - 1) / threads;
     if (blocks > 148 * 8) blocks = 148 * 8;
-    sw_kv_append_kernel<<<(unsigned)blocks, threads, 0, stream>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, sw_kv_append_kernel, p);
 }
 
 // ---------------------------------------------------------------------------------------------------------------
@@ -413,24 +426,34 @@ __device__ bool run_unit(const CUtensorMap* kv_map, const MixedParams& p, const 
     __threadfence();
     if (lane == 0) p.tickets[u.ticket] = 0;  // ready for the next launch
     const int slot0 = u.slot - u.split * p.Hkv;
+    const int ns = u.nsplit;
     for (int r = 0; r < g; ++r) {
+        // running maximum and weighted sum over the splits: lanes take splits, then one warp reduction each
+        const float* ml = p.part_ml + (int64_t)slot0 * (2 * kMaxGroup) + r;   // split s: + s * ml_stride
+        const int64_t ml_stride = (int64_t)p.Hkv * (2 * kMaxGroup);
         float m_all = -INFINITY;
-#pragma unroll 4
-        for (int sidx = 0; sidx < u.nsplit; ++sidx)
-            m_all = fmaxf(m_all, __ldcg(&p.part_ml[(int64_t)(slot0 + sidx * p.Hkv) * (2 * kMaxGroup) + r]));
+        for (int sidx = lane; sidx < ns; sidx += 32) m_all = fmaxf(m_all, __ldcg(ml + sidx * ml_stride));
+#pragma unroll
+        for (int o2 = 16; o2 > 0; o2 >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xffffffffu, m_all, o2));
         float l_all = 0.f;
+        for (int sidx = lane; sidx < ns; sidx += 32) {
+            const float ms = __ldcg(ml + sidx * ml_stride);
+            l_all += (ms == -INFINITY ? 0.f : fast_exp2((ms - m_all) * p.sm_scale_log2)) * __ldcg(ml + sidx * ml_stride + kMaxGroup);
+        }
+#pragma unroll
+        for (int o2 = 16; o2 > 0; o2 >>= 1) l_all += __shfl_xor_sync(0xffffffffu, l_all, o2);
+        // weighted sum of the partial outputs: lanes take columns, eight splits' loads in flight
         float acc[D / 32];
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) acc[c] = 0.f;
-#pragma unroll 4
-        for (int sidx = 0; sidx < u.nsplit; ++sidx) {
-            const int64_t sl = slot0 + sidx * p.Hkv;
-            const float ms = __ldcg(&p.part_ml[sl * (2 * kMaxGroup) + r]);
-            const float ls = __ldcg(&p.part_ml[sl * (2 * kMaxGroup) + kMaxGroup + r]);
-            const float w = fast_exp2((ms - m_all) * p.sm_scale_log2);
-            l_all += ls * w;
+        const float* po = p.part_o + ((int64_t)slot0 * g + r) * D + lane;      // split s: + s * po_stride
+        const int64_t po_stride = (int64_t)p.Hkv * g * D;
+#pragma unroll 8
+        for (int sidx = 0; sidx < ns; ++sidx) {
+            const float ms = __ldcg(ml + sidx * ml_stride);
+            const float w = ms == -INFINITY ? 0.f : fast_exp2((ms - m_all) * p.sm_scale_log2);
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) acc[c] += w * __ldcg(&p.part_o[(sl * g + r) * D + c * 32 + lane]);
+            for (int c = 0; c < D / 32; ++c) acc[c] = fmaf(w, __ldcg(po + sidx * po_stride + c * 32), acc[c]);
         }
         const float inv = 1.f / l_all;
         const int hd = u.kvh * g + r;
@@ -476,6 +499,10 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
         misc[1] = 0;
         fence_mbar_init();
     }
+    // Everything above touched only shared memory and kernel parameters.  From here on the kernel reads what earlier
+    // kernels of the stream wrote (the pool after the KV append, q, the page tables): wait for them to finish.
+    grid_dependency_wait();
+    grid_launch_dependents();
     __syncthreads();
 
     // chunk-prefill tiles first (long, tensor-bound); the decode units below fill the tail
@@ -599,12 +626,18 @@ cudaError_t configure_kernels(int head_dim) {
 
 cudaError_t launch_mixed_attn(int head_dim, const CUtensorMap& kv_map, const CUtensorMap& q_map, const MixedParams& p,
                               int num_sms, cudaStream_t stream) {
-    const size_t smem = mixed_attn_smem_bytes(head_dim);
-    if (head_dim == 64)
-        sw_mixed_attn_kernel<64><<<num_sms, kThreads, smem, stream>>>(kv_map, q_map, p);
-    else
-        sw_mixed_attn_kernel<128><<<num_sms, kThreads, smem, stream>>>(kv_map, q_map, p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)num_sms);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = mixed_attn_smem_bytes(head_dim);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // prologue overlaps the previous kernel's tail
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (head_dim == 64) return cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<64>, kv_map, q_map, p);
+    return cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<128>, kv_map, q_map, p);
 }
 
 }  // namespace sw

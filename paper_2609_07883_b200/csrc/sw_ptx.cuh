@@ -43,6 +43,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     return true;
 }
 
+// ---- programmatic dependent launch --------------------------------------------------------------------------
+// grid_dependency_wait: block until the kernels this launch depends on have finished and their writes are visible
+// (a no-op when the launch carries no programmatic dependency).  grid_launch_dependents: let the next kernel in the
+// stream begin its own prologue.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- proxy fences -----------------------------------------------------------------------------------------
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
