@@ -90,3 +90,115 @@ def to_cost_table(table: dict, interp: bool = False, which: str = "p99_ns"):
 
     return B.CostTable(table["n_grid"], table["ctx_grid"], table["prefix_grid"], table["chunk_grid"],
                        np.asarray(table[which], dtype=np.int64), make_monotone=True, interp=interp)
+
+
+# --------------------------------------------------------------------------------------------------------------------
+# cost-surface sweeps of the named workloads (command line)
+# --------------------------------------------------------------------------------------------------------------------
+NOMINAL_HBM_GBS = 8000.0
+NOMINAL_BF16_TFLOPS = 2250.0
+
+
+def _work(batch: W.MixedBatch) -> dict:
+    sh = batch.shape
+    P, C, n, ctx = batch.prefix_len, batch.chunk_len, batch.num_decode, batch.total_decode_ctx
+    qo_row = sh.num_q_heads * sh.head_dim * 2 * 2
+    return {"decode_bytes": ctx * sh.token_bytes + n * qo_row,
+            "prefill_bytes": ((P + C) * sh.token_bytes if C else 0) + C * qo_row,
+            "prefill_flops": 4 * sh.num_q_heads * sh.head_dim * (C * P + C * (C + 1) // 2)}
+
+
+def sweep(config: str, reps: int, log) -> list:
+    """Mixed, prefill-only and decode-only launch times over the workload's (prefix, chunk) grid."""
+    import json as _json
+
+    import torch
+
+    from . import binding as B
+
+    peaks_file = Path(__file__).resolve().parent.parent / "MEASURED_PEAKS.json"
+    peaks = _json.loads(peaks_file.read_text()) if peaks_file.exists() else {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
+    dev = torch.device("cuda", 0)
+    shape = W.LLAMA
+    if config == "chat":
+        grid = [(512, c, n) for n in (16, 64) for c in (64, 128, 256, 512)]
+        make = lambda P, C, n: W.chat_batch(n=n, chunk_len=C, prefix_len=P, rng=W.rng_for(1))
+        layers, pool_pages = 8, None
+    elif config == "mixed":
+        grid = [(P, c, 128) for P in (0, 4096, 16384, 28672) for c in (64, 128, 256, 512, 1024, 2048, 4096)]
+        make = lambda P, C, n: W.mixed_batch(C, P, n=n, rng=W.rng_for(2))
+        layers, pool_pages = 2, None
+    else:
+        grid = [(98304, c, 16) for c in (1024, 4096, 8192)]
+        free, _ = torch.cuda.mem_get_info()
+        pool_pages = int(min(120e9, 0.9 * free) // (shape.page_elems * 2))   # ~120 GB pool, live pages scattered over it
+        make = lambda P, C, n: W.long_batch(C, P, n=n, num_pages=pool_pages, rng=W.rng_for(3))
+        layers = 1
+    rows = []
+    pools, pool_size = [], 0
+    for (P, C, n) in grid:
+        batch = make(P, C, n)
+        if batch.num_pages != pool_size:
+            pools, pool_size = [], batch.num_pages
+            torch.cuda.empty_cache()
+            for layer in range(layers):
+                t = torch.empty(batch.num_pages * shape.page_elems, dtype=torch.bfloat16, device=dev)
+                W.fill_normal_bf16_(t, W.SEED_BASE + 500 + layer)
+                pools.append(t)
+        total_pages = int(batch.prefill_pages.shape[0] + batch.decode_pages.shape[0])
+        ctx = B.Context(shape, batch.num_pages, max(C, 1), max(n, 1), total_pages + 16)
+        q = torch.randn(batch.num_rows, shape.num_q_heads, shape.head_dim, device=dev).to(torch.bfloat16)
+        out = torch.empty_like(q)
+        variants = {"mixed": batch,
+                    "prefill_only": W.MixedBatch(shape, batch.num_pages, P, C, batch.prefill_pages, np.zeros(0, np.int32),
+                                                 np.zeros(1, np.int32), np.zeros(0, np.int32)),
+                    "decode_only": W.MixedBatch(shape, batch.num_pages, 0, 0, np.zeros(0, np.int32), batch.decode_kv_len,
+                                                batch.decode_page_indptr, batch.decode_pages)}
+        row = {"prefix": P, "chunk": C, "decodes": n, "decode_ctx": batch.total_decode_ctx, "pool_pages": batch.num_pages}
+        w = _work(batch)
+        for name, b in variants.items():
+            db = B.DeviceBatch(b, dev)
+            qq = q if name != "decode_only" else q[C:]
+            p50, p99, _ = B.sw_cost_probe(ctx, pools, db, qq, out[: b.num_rows], warmup=2, reps=reps)
+            row[name + "_us_p50"] = p50 / 1e3 / layers
+            row[name + "_us_p99"] = p99 / 1e3 / layers
+        B.sw_check_status(ctx)
+        t_pf, t_dec, t_mix = (row[k + "_us_p50"] * 1e-6 for k in ("prefill_only", "decode_only", "mixed"))
+        row["prefill_tflops"] = w["prefill_flops"] / t_pf / 1e12
+        row["prefill_frac_measured"] = row["prefill_tflops"] / peaks["bf16_tflops"]
+        row["prefill_frac_nominal"] = row["prefill_tflops"] / NOMINAL_BF16_TFLOPS
+        row["decode_gbs"] = w["decode_bytes"] / t_dec / 1e9
+        row["decode_frac_measured"] = row["decode_gbs"] / peaks["hbm_gbs"]
+        row["decode_frac_nominal"] = row["decode_gbs"] / NOMINAL_HBM_GBS
+        row["prefill_tokens_per_s"] = C / t_mix
+        row["decode_tokens_per_s"] = n / t_mix
+        row["mixed_vs_sum"] = t_mix / (t_pf + t_dec)
+        rows.append(row)
+        log(f"P={P:6d} C={C:5d} n={n:4d}  mixed {row['mixed_us_p50']:9.1f} us  prefill {row['prefill_only_us_p50']:9.1f} us "
+            f"({row['prefill_tflops']:7.1f} TFLOP/s, {row['prefill_frac_measured']:.2f} of measured, "
+            f"{row['prefill_frac_nominal']:.2f} of nominal)  decode {row['decode_only_us_p50']:8.1f} us ({row['decode_gbs']:6.0f} GB/s, "
+            f"{row['decode_frac_measured']:.2f} / {row['decode_frac_nominal']:.2f})  mixed/(pf+dec) {row['mixed_vs_sum']:.2f}")
+        del ctx
+    return rows
+
+
+def main(argv=None):
+    import argparse
+    import sys
+
+    from . import build
+
+    ap = argparse.ArgumentParser(description="cost surface of a named workload: mixed / prefill-only / decode-only launches")
+    ap.add_argument("--config", choices=["chat", "mixed", "long"], default="mixed")
+    ap.add_argument("--reps", type=int, default=10)
+    ap.add_argument("--out", default=None)
+    args = ap.parse_args(argv)
+    build.build()
+    rows = sweep(args.config, args.reps, lambda s: print(s, flush=True))
+    out = args.out or f"gpurun_out/cost_surface_{args.config}.json"
+    Path(out).parent.mkdir(parents=True, exist_ok=True)
+    Path(out).write_text(json.dumps(rows, indent=1))
+
+
+if __name__ == "__main__":
+    main()
