@@ -24,9 +24,11 @@ struct PfGeo {
     static constexpr int kPageBytes = kPageSize * 128;           // one page's rows inside a half
 };
 
+// P of a tile is handed to the MMA warp in two halves (keys 0-63, then 64-127) so that the first four P V
+// instructions run while the second half is still being exponentiated.
 enum PfBar {
     kBarQFull = 0, kBarKFull = 1, kBarVLanded = 3, kBarVFull = 5, kBarKEmpty = 7, kBarVEmpty = 9,
-    kBarSFull = 11, kBarPFull = 13, kBarODone = 15, kPfBars = 17
+    kBarSFull = 11, kBarPHalf = 13 /* [tile][half] */, kBarODone = 17, kPfBars = 19
 };
 
 // register budgets per warpgroup during the prefill phase: 128 * 72 + 256 * 216 <= 384 * 168
@@ -40,7 +42,7 @@ struct PfShared {
 };
 
 __device__ __forceinline__ void pf_init_barriers(uint32_t bars) {
-    for (int i = 0; i < kPfBars; ++i) mbar_init(bars + i * 8, (i == kBarPFull || i == kBarPFull + 1) ? 4 : 1);
+    for (int i = 0; i < kPfBars; ++i) mbar_init(bars + i * 8, (i >= kBarPHalf && i < kBarPHalf + 4) ? 4 : 1);
 }
 
 // Bounded wait that also gives up when another role of this CTA has given up.
@@ -242,44 +244,59 @@ struct PfMmaState {
     uint32_t p_cnt[2] = {0, 0};
 };
 
+// The whole MMA warp runs this role in lockstep (waits included) so that addresses and descriptors stay in uniform
+// registers; only the tcgen05.mma / tcgen05.commit instructions themselves are issued by the one elected lane.
 template <int D>
-__device__ __forceinline__ void pf_issue_qk(const PfShared& sh, int t, uint32_t s) {
+__device__ __forceinline__ void pf_issue_qk(const PfShared& sh, int t, uint32_t s, bool leader) {
     using G = PfGeo<D>;
     constexpr uint32_t idesc = umma_idesc_bf16(128, 128, 0, 0);
-    const uint32_t q = sh.smem + G::kQOffset + t * G::kTileBytes;
-    const uint32_t k = sh.smem + G::kKVOffset + s * 2 * G::kTileBytes;
+    const uint64_t qd = umma_desc_sw128(sh.smem + G::kQOffset + t * G::kTileBytes, 16, 1024);
+    const uint64_t kd = umma_desc_sw128(sh.smem + G::kKVOffset + s * 2 * G::kTileBytes, 16, 1024);
+    const uint32_t d_tmem = sh.tmem + t * 128;
+    if (leader) {
 #pragma unroll
-    for (int ks = 0; ks < D / 16; ++ks) {
-        const uint32_t off = (ks >> 2) * G::kHalfBytes + (ks & 3) * 32;
-        tc_mma_ss(sh.tmem + t * 128, umma_desc_sw128(q + off, 16, 1024), umma_desc_sw128(k + off, 16, 1024), idesc, ks > 0);
+        for (int ks = 0; ks < D / 16; ++ks) {
+            const uint64_t off = (uint64_t)(((ks >> 2) * G::kHalfBytes + (ks & 3) * 32) >> 4);  // descriptor address units
+            tc_mma_ss(d_tmem, qd + off, kd + off, idesc, ks > 0);
+        }
+        tc_commit(sh.bars + (kBarSFull + t) * 8);
     }
-    tc_commit(sh.bars + (kBarSFull + t) * 8);
 }
 
+// one half of O_t += P_t V: keys [64 * half, 64 * half + 64), 16 keys per instruction
 template <int D>
-__device__ __forceinline__ void pf_issue_pv(const PfShared& sh, int t, uint32_t s, bool first) {
+__device__ __forceinline__ void pf_issue_pv_half(const PfShared& sh, int t, uint32_t s, int half, bool first, bool leader) {
     using G = PfGeo<D>;
     constexpr uint32_t idesc = umma_idesc_bf16(128, D, 0, 1);  // B = V is MN-major: [key][d] with d contiguous
-    const uint32_t v = sh.smem + G::kKVOffset + s * 2 * G::kTileBytes + G::kTileBytes;
+    const uint64_t vd = umma_desc_sw128(sh.smem + G::kKVOffset + s * 2 * G::kTileBytes + G::kTileBytes + half * 4 * 2048,
+                                        G::kHalfBytes, 1024);
+    const uint32_t d_tmem = sh.tmem + 256 + t * D;
+    const uint32_t p_tmem = sh.tmem + t * 128 + half * 32;
+    const uint32_t acc_first = first && half == 0 ? 0u : 1u;
+    if (leader) {
 #pragma unroll
-    for (int ks = 0; ks < 8; ++ks)  // 16 keys per instruction
-        tc_mma_ts(sh.tmem + 256 + t * D, sh.tmem + t * 128 + ks * 8, umma_desc_sw128(v + ks * 2 * 1024, G::kHalfBytes, 1024),
-                  idesc, !(first && ks == 0));
-    tc_commit(sh.bars + (kBarODone + t) * 8);
+        for (int i = 0; i < 4; ++i)
+            tc_mma_ts(d_tmem, p_tmem + i * 8, vd + (uint64_t)(i * (2048 >> 4)), idesc, i == 0 ? acc_first : 1u);
+        if (half == 1) tc_commit(sh.bars + (kBarODone + t) * 8);
+    }
 }
 
 template <int D>
 __device__ __forceinline__ bool pf_mma(const MixedParams& p, const PfShared& sh, const PfItem& it, PfMmaState& st) {
+    const bool leader = elect_one();
     auto act = [&](int t, int j) { return j < it.j1 && j < it.nkv[t]; };
     auto last_active = [&](int j) { return act(1, j) ? 1 : 0; };
+    auto commit = [&](int bar) {
+        if (leader) tc_commit(sh.bars + bar * 8);
+    };
     if (!pf_wait(sh, kBarQFull, st.q_it & 1, p.ctrl, 4)) return false;
     {
         const uint32_t s = st.kv_it & 1, n = st.kv_it >> 1;
         if (!pf_wait(sh, kBarKFull + s, n & 1, p.ctrl, 5)) return false;
         tc_fence_after_sync();
         for (int t = 0; t < 2; ++t)
-            if (act(t, it.j0)) pf_issue_qk<D>(sh, t, s);
-        tc_commit(sh.bars + (kBarKEmpty + s) * 8);
+            if (act(t, it.j0)) pf_issue_qk<D>(sh, t, s, leader);
+        commit(kBarKEmpty + s);
     }
     for (int j = it.j0; j < it.j1; ++j) {
         const uint32_t cur = st.kv_it + (j - it.j0);
@@ -289,20 +306,22 @@ __device__ __forceinline__ bool pf_mma(const MixedParams& p, const PfShared& sh,
         bool k_ready = false;  // K of tile j+1 is awaited as late as possible: right before its first use
         for (int t = 0; t < 2; ++t) {
             if (act(t, j)) {
-                if (!pf_wait(sh, kBarPFull + t, st.p_cnt[t] & 1, p.ctrl, 8)) return false;
+                for (int half = 0; half < 2; ++half) {
+                    if (!pf_wait(sh, kBarPHalf + 2 * t + half, st.p_cnt[t] & 1, p.ctrl, 8)) return false;
+                    tc_fence_after_sync();
+                    pf_issue_pv_half<D>(sh, t, s, half, j == it.j0, leader);
+                }
                 st.p_cnt[t] += 1;
-                tc_fence_after_sync();
-                pf_issue_pv<D>(sh, t, s, j == it.j0);
             }
-            if (t == last_active(j)) tc_commit(sh.bars + (kBarVEmpty + s) * 8);
+            if (t == last_active(j)) commit(kBarVEmpty + s);
             if (act(t, j + 1)) {
                 if (!k_ready) {
                     if (!pf_wait(sh, kBarKFull + (s ^ 1), ((cur + 1) >> 1) & 1, p.ctrl, 7)) return false;
                     k_ready = true;
                 }
-                pf_issue_qk<D>(sh, t, s ^ 1);
+                pf_issue_qk<D>(sh, t, s ^ 1, leader);
             }
-            if (more && t == last_active(j + 1)) tc_commit(sh.bars + (kBarKEmpty + (s ^ 1)) * 8);
+            if (more && t == last_active(j + 1)) commit(kBarKEmpty + (s ^ 1));
         }
     }
     st.kv_it += it.j1 - it.j0;
@@ -438,6 +457,12 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
                 pk[i] = pack_bf16x2(p0, p1);
             }
             tmem_st_32x32b_x16(s_addr + c * 16, pk);
+            if (c == 1) {  // the first 64 keys of P are in place: the first half of P V may start
+                tc_wait_st();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(sh.bars + (kBarPHalf + 2 * t) * 8);
+            }
         }
         {
             float a0, a1, b0, b1;
@@ -448,7 +473,7 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
         tc_wait_st();
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(sh.bars + (kBarPFull + t) * 8);
+        if (lane == 0) mbar_arrive(sh.bars + (kBarPHalf + 2 * t + 1) * 8);
     }
 
     // the piece's O is complete once its last P V has been committed
@@ -594,7 +619,7 @@ __device__ __forceinline__ void prefill_phase(const CUtensorMap* kv_map, const C
             if (warp == 0) {
                 if (lane == 0 && it.j1 > it.j0) pf_produce<D>(kv_map, q_map, p, sh, it, prod_kv_it);
             } else if (warp == 1) {
-                if (lane == 0 && it.j1 > it.j0) pf_mma<D>(p, sh, it, mma_state);
+                if (it.j1 > it.j0) pf_mma<D>(p, sh, it, mma_state);
             } else if (warp == 2) {
                 if (it.j1 > it.j0) pf_sanitize<D>(p, sh, it, san_kv_it);
             } else {
