@@ -165,47 +165,48 @@ __device__ __forceinline__ PfItem pf_entry(const MixedParams& p, const PfPlan& p
     return it;
 }
 
-// ---- role: TMA producer (one thread) ---------------------------------------------------------------------------
+// ---- role: TMA producer (one warp) ----------------------------------------------------------------------------
 template <int D>
 __device__ __forceinline__ bool pf_produce(const CUtensorMap* kv_map, const CUtensorMap* q_map, const MixedParams& p,
                                            const PfShared& sh, const PfItem& it, uint32_t& kv_it) {
     using G = PfGeo<D>;
-    const int tt = 128 / p.group;
+    // The whole warp runs the role: lane i owns page i of every 128-key tile (its page id, its TMA boxes), so the
+    // eight pages of a tile are issued by one instruction instead of a loop of one thread.
+    const int lane = threadIdx.x & 31;
     // Q tiles (rows past the chunk are zero-filled by the tensor map's bounds)
-    int active = (it.nkv[0] > it.j0) + (it.nkv[1] > it.j0);
-    mbar_arrive_expect_tx(sh.bars + kBarQFull * 8, active * G::kTileBytes);
-    for (int t = 0; t < 2; ++t)
-        if (it.nkv[t] > it.j0)
-            for (int h = 0; h < G::kHalves; ++h)
-                tma_load_3d(sh.smem + G::kQOffset + t * G::kTileBytes + h * G::kHalfBytes, q_map, sh.bars + kBarQFull * 8,
-                            h * 64, it.kvh * p.group, it.tok0[t]);
-    (void)tt;
+    if (lane == 0) {
+        const int active = (it.nkv[0] > it.j0) + (it.nkv[1] > it.j0);
+        mbar_arrive_expect_tx(sh.bars + kBarQFull * 8, active * G::kTileBytes);
+        for (int t = 0; t < 2; ++t)
+            if (it.nkv[t] > it.j0)
+                for (int h = 0; h < G::kHalves; ++h)
+                    tma_load_3d(sh.smem + G::kQOffset + t * G::kTileBytes + h * G::kHalfBytes, q_map, sh.bars + kBarQFull * 8,
+                                h * 64, it.kvh * p.group, it.tok0[t]);
+    }
     const int npages = (p.P + p.C + kPageSize - 1) / kPageSize;
+    auto page_of = [&](int j) { return (lane < 8 && j * 8 + lane < npages) ? p.prefill_pages[j * 8 + lane] : 0; };
+    int id_next = page_of(it.j0);
     for (int j = it.j0; j < it.j1; ++j, ++kv_it) {
         const uint32_t s = kv_it & 1, n = kv_it >> 1;
-        const int pg0 = j * 8;
-        const int nvp = min(8, npages - pg0);
-        int ids[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) ids[i] = i < nvp ? p.prefill_pages[pg0 + i] : 0;
+        const int id = id_next;
+        if (j + 1 < it.j1) id_next = page_of(j + 1);  // in flight while this tile is issued
+        const int nvp = min(8, npages - j * 8);
         const uint32_t kdst = sh.smem + G::kKVOffset + s * 2 * G::kTileBytes;
         const uint32_t vdst = kdst + G::kTileBytes;
         if (!pf_wait(sh, kBarKEmpty + s, (n & 1) ^ 1, p.ctrl, 1)) return false;
-        mbar_arrive_expect_tx(sh.bars + (kBarKFull + s) * 8, nvp * G::kHalves * G::kPageBytes);
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-            if (i < nvp)
-                for (int h = 0; h < G::kHalves; ++h)
-                    tma_load_4d(kdst + h * G::kHalfBytes + i * G::kPageBytes, kv_map, sh.bars + (kBarKFull + s) * 8, h * 64, 0,
-                                it.kvh, ids[i]);
+        if (lane == 0) mbar_arrive_expect_tx(sh.bars + (kBarKFull + s) * 8, nvp * G::kHalves * G::kPageBytes);
+        __syncwarp();
+        if (lane < nvp)
+            for (int h = 0; h < G::kHalves; ++h)
+                tma_load_4d(kdst + h * G::kHalfBytes + lane * G::kPageBytes, kv_map, sh.bars + (kBarKFull + s) * 8, h * 64, 0,
+                            it.kvh, id);
         if (!pf_wait(sh, kBarVEmpty + s, (n & 1) ^ 1, p.ctrl, 2)) return false;
-        mbar_arrive_expect_tx(sh.bars + (kBarVLanded + s) * 8, nvp * G::kHalves * G::kPageBytes);
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-            if (i < nvp)
-                for (int h = 0; h < G::kHalves; ++h)
-                    tma_load_4d(vdst + h * G::kHalfBytes + i * G::kPageBytes, kv_map, sh.bars + (kBarVLanded + s) * 8, h * 64,
-                                0, p.Hkv + it.kvh, ids[i]);
+        if (lane == 0) mbar_arrive_expect_tx(sh.bars + (kBarVLanded + s) * 8, nvp * G::kHalves * G::kPageBytes);
+        __syncwarp();
+        if (lane < nvp)
+            for (int h = 0; h < G::kHalves; ++h)
+                tma_load_4d(vdst + h * G::kHalfBytes + lane * G::kPageBytes, kv_map, sh.bars + (kBarVLanded + s) * 8, h * 64, 0,
+                            p.Hkv + it.kvh, id);
     }
     return true;
 }
@@ -617,7 +618,7 @@ __device__ __forceinline__ void prefill_phase(const CUtensorMap* kv_map, const C
         for (int iter = 0; entry < plan.n_entries; ++iter) {
             const PfItem it = pf_entry(p, plan, entry);
             if (warp == 0) {
-                if (lane == 0 && it.j1 > it.j0) pf_produce<D>(kv_map, q_map, p, sh, it, prod_kv_it);
+                if (it.j1 > it.j0) pf_produce<D>(kv_map, q_map, p, sh, it, prod_kv_it);
             } else if (warp == 1) {
                 if (it.j1 > it.j0) pf_mma<D>(p, sh, it, mma_state);
             } else if (warp == 2) {
