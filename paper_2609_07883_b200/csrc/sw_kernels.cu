@@ -219,18 +219,20 @@ struct WarpRing {
     uint32_t it;    // pages consumed so far (stage = it % kStages, parity = (it / kStages) & 1)
 };
 
+// Whole-warp call: lane 0 arms the stage's barrier, lanes 0 .. 2*halves-1 each issue one of the page's boxes.
 template <int D>
 __device__ __forceinline__ void issue_page(const CUtensorMap* kv_map, const WarpRing<D>& ring, uint32_t issue_it, int page,
                                            int kvh, int Hkv) {
+    const int lane = threadIdx.x & 31;
     const uint32_t stage = issue_it % kStages;
     const uint32_t dst = ring.buf + stage * Geo<D>::kStageBytes;
     const uint32_t bar = ring.bar + stage * 8;
-    mbar_arrive_expect_tx(bar, Geo<D>::kStageBytes);
-#pragma unroll
-    for (int x = 0; x < 2; ++x)
-#pragma unroll
-        for (int h = 0; h < Geo<D>::kHalves; ++h)
-            tma_load_4d(dst + (x * Geo<D>::kHalves + h) * Geo<D>::kBlockBytes, kv_map, bar, h * 64, 0, x * Hkv + kvh, page);
+    if (lane == 0) mbar_arrive_expect_tx(bar, Geo<D>::kStageBytes);
+    __syncwarp();
+    if (lane < 2 * Geo<D>::kHalves) {
+        const int x = lane / Geo<D>::kHalves, h = lane % Geo<D>::kHalves;
+        tma_load_4d(dst + lane * Geo<D>::kBlockBytes, kv_map, bar, h * 64, 0, x * Hkv + kvh, page);
+    }
 }
 
 // Runs one unit; returns false if a bounded wait expired.
@@ -286,7 +288,7 @@ __device__ bool run_unit(const CUtensorMap* kv_map, const MixedParams& p, const 
         if (page < 0 || (int64_t)page >= p.num_pages) {
             if (lane == 0) report(p.ctrl, SW_ERR_OUT_OF_RANGE, kSiteAttnPage, u.q_row);
         }
-        if (lane == 0) issue_page<D>(kv_map, ring, it0 + issued, page, u.kvh, p.Hkv);
+        issue_page<D>(kv_map, ring, it0 + issued, page, u.kvh, p.Hkv);
         ++issued;
     };
     for (int k = 0; k < kStages && k < npg; ++k) issue_next();
