@@ -27,6 +27,9 @@ sys.path.insert(0, str(ROOT))
 
 from paper_2609_07883_b200 import workloads as W  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one sw_mixed_attn_kernel<128> launch of the default workload, from the
+# ncu capture summarised in profiles/sw_mixed_attn_kernel_chat_bench.md (298.6 MB read + 11.0 MB written)
+NCU_TRAFFIC_DEFAULT_WORKLOAD = 309_597_952
 NOMINAL_HBM_GBS = 8000.0
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -334,6 +337,8 @@ def run_ours(args) -> dict:
     us = ms_total / args.steps * 1e3
     peaks, peak_kind = measured_peaks()
     achieved_gbs = work["attn_bytes"] / (attn_ms * 1e-3) / 1e9
+    is_default = (args.workload, args.decodes, args.chunk, args.prefix) == ("chat",) + WORKLOAD_DEFAULTS["chat"]
+    traffic = NCU_TRAFFIC_DEFAULT_WORKLOAD if is_default else None
     result = {
         "metric": "mixed_iteration_us", "value": us, "unit": "us", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": False, "scaling": "weak",
@@ -343,7 +348,7 @@ def run_ours(args) -> dict:
         "decode_tokens_per_s": agg["decode_tokens_per_s"],
         "attn_launch_us": attn_ms * 1e3,
         "roofline": {"bound": "hbm", "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved_gbs / peaks["hbm_gbs"], "traffic": None, "peak_kind": f"of {peak_kind}",
+                     "frac": achieved_gbs / peaks["hbm_gbs"], "traffic": traffic, "peak_kind": f"of {peak_kind}",
                      "kernel": "sw_mixed_attn_kernel<128>", "algorithmic_bytes_per_launch": work["attn_bytes"],
                      "frac_of_nominal_8TBs": achieved_gbs / NOMINAL_HBM_GBS,
                      "prefill_tflops": work["prefill_flops"] / (attn_ms * 1e-3) / 1e12},
