@@ -283,14 +283,15 @@ def run_ours(args) -> dict:
     def reduce_max(x: float) -> float:
         return reduce_max_over_ranks(x, dev)
 
+    # clocks are sampled from before the warm-up to after the last timed loop (nvidia-smi needs a moment to start)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.4)
     for i in range(args.warmup):
         step(i)
     sync_all()
     B.sw_check_status(ctx)
-
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
     # (1) the timed region: K steps, device-timed
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sync_all()
@@ -369,8 +370,8 @@ def run_ours(args) -> dict:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="chat", choices=sorted(WORKLOAD_DEFAULTS))
     ap.add_argument("--decodes", type=int, default=None)
