@@ -73,7 +73,6 @@ _lib.sw_cost_table_lookup.argtypes = [_vp, _i64, _i64, _i64, _i64, C.POINTER(_i6
 _lib.sw_choose_chunk.argtypes = [_vp, C.POINTER(sw_chooser_params), _i64, C.POINTER(_i64), _i32, _i64, _i32, _i32,
                                  C.POINTER(sw_choice)]
 _lib.sw_last_error.restype = C.c_char_p
-_lib.sw_debug_set_prefill_rows.argtypes = [_vp, C.c_int]
 
 
 class SwError(RuntimeError):
@@ -221,8 +220,6 @@ def sw_decode_attn_static(layout: sw_layout, device: int, kv_pool, batch: Device
                                       _ptr(lse), _stream_handle(stream)), "sw_decode_attn_static")
 
 
-def sw_debug_set_prefill_rows(ctx: Context, on: bool) -> None:
-    _lib.sw_debug_set_prefill_rows(ctx.handle, int(on))
 
 
 # ---------------------------------------------------------------------------------------------------------------

@@ -80,7 +80,6 @@ struct sw_ctx {
     };
     std::vector<MapEntry> kv_maps;  // small cache: one entry per pool of a layer stack
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-    int bringup_prefill_rows = 0;
 };
 
 namespace {
@@ -271,11 +270,10 @@ sw_status sw_mixed_attn_run(sw_ctx* ctx, const void* kv_pool, const sw_batch* ba
     p.pf_ml = reinterpret_cast<float*>(ctx->ws + ctx->w.pf_ml);
     p.pf_o = reinterpret_cast<float*>(ctx->ws + ctx->w.pf_o);
     p.pf_tickets = reinterpret_cast<int32_t*>(ctx->ws + ctx->w.pf_tickets);
-    p.prefill_rows_on_decode_path = ctx->bringup_prefill_rows;
     // q as [row][head][element] restricted to the chunk rows: one box = 128 tile rows (token-major, the g heads of a
     // KV head minor) x 64 elements; rows past the chunk read as zero
     CUtensorMap q_map = *kv_map;
-    if (p.C > 0 && !p.prefill_rows_on_decode_path) {
+    if (p.C > 0) {
         const cuuint64_t dims[3] = {(cuuint64_t)l.head_dim, (cuuint64_t)l.num_q_heads, (cuuint64_t)p.C};
         const cuuint64_t strides[2] = {(cuuint64_t)l.head_dim * 2, (cuuint64_t)l.num_q_heads * l.head_dim * 2};
         const cuuint32_t box[3] = {64, (cuuint32_t)p.group, (cuuint32_t)(128 / p.group)};
@@ -389,13 +387,6 @@ sw_status sw_check_status(sw_ctx* ctx, void* stream, int32_t* code, int32_t* det
     if (words[0] != 0)
         return sw_fail((sw_status)words[0], "device reported status %d at site %d index %d", words[0], (words[1] >> 24) & 0xFF,
                        words[1] & 0xFFFFFF);
-    return SW_OK;
-}
-
-// Bring-up switch (not part of the public header): 1 runs every chunk row as a one-token unit of the decode path.
-sw_status sw_debug_set_prefill_rows(sw_ctx* ctx, int on) {
-    if (!ctx) return SW_ERR_INVALID_ARG;
-    ctx->bringup_prefill_rows = on;
     return SW_OK;
 }
 

@@ -53,7 +53,6 @@ struct MixedParams {
     float* pf_ml;        // [kMaxCtas][2][2][128]
     float* pf_o;         // [kMaxCtas][2][128][D]
     int32_t* pf_tickets; // [items][2]
-    int prefill_rows_on_decode_path;  // bring-up switch: run every chunk row as a one-token unit
 };
 
 struct AppendParams {

@@ -117,7 +117,6 @@ struct Geo {
 struct Plan {
     int split_tokens;   // tokens per split-KV unit (multiple of the page size)
     int decode_units;   // sum over requests of ceil(len / split_tokens)
-    int prefill_items;  // chunk-row units on the decode path (bring-up)
     int total_items;
 };
 
@@ -192,8 +191,7 @@ __device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix
     if (threadIdx.x == 0) unit_prefix[p.n] = total_units;
     __syncthreads();
     plan.decode_units = total_units;
-    plan.prefill_items = p.prefill_rows_on_decode_path ? p.C * p.Hkv : 0;
-    plan.total_items = plan.prefill_items + total_units * p.Hkv;
+    plan.total_items = total_units * p.Hkv;
     return plan;
 }
 
@@ -488,7 +486,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     int* unit_prefix = reinterpret_cast<int*>(smem + Geo<D>::kPlanOffset);
     int* scratch = reinterpret_cast<int*>(smem + Geo<D>::kMiscOffset);
 
-    const bool tensor_prefill = p.C > 0 && !p.prefill_rows_on_decode_path;
+    const bool tensor_prefill = p.C > 0;
     volatile int* misc = reinterpret_cast<volatile int*>(scratch + 32);  // [0] TMEM base, [1] abort flag, [2..3] ticket flags
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&kv_map);
@@ -540,7 +538,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     }
 
     const Plan plan = make_plan(p, unit_prefix, scratch);
-    if (plan.total_items > p.max_items + plan.prefill_items) {
+    if (plan.total_items > p.max_items) {
         if (threadIdx.x == 0) report(p.ctrl, SW_ERR_WORKSPACE, kSiteScratch, plan.total_items);
     } else {
         WarpRing<D> ring;
@@ -554,21 +552,8 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
             if (item >= plan.total_items) break;
             Unit u;
             bool ok = true;
-            if (item < plan.prefill_items) {
-                const int j = item / p.Hkv;
-                u.q_row = j;
-                u.kvh = item % p.Hkv;
-                u.len = p.P + j + 1;
-                u.t_begin = 0;
-                u.t_end = u.len;
-                u.nsplit = 1;
-                u.split = 0;
-                u.ticket = 0;
-                u.slot = 0;
-                u.pages = p.prefill_pages;
-                ok = (u.len + kPageSize - 1) / kPageSize <= p.num_prefill_pages;
-            } else {
-                const int di = item - plan.prefill_items;
+            {
+                const int di = item;
                 const int unit = di / p.Hkv;
                 u.kvh = di % p.Hkv;
                 int lo = 0, hi = p.n;  // largest i with unit_prefix[i] <= unit

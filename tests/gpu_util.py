@@ -25,7 +25,7 @@ def torch_to_bits(t) -> np.ndarray:
 class Runner:
     """Device buffers for one batch; runs append + attention through the binding."""
 
-    def __init__(self, batch: W.MixedBatch, tensors: dict, device=0, prefill_rows: bool | None = None):
+    def __init__(self, batch: W.MixedBatch, tensors: dict, device=0):
         import torch
         from paper_2609_07883_b200 import binding as B
 
@@ -36,8 +36,6 @@ class Runner:
         total_pages = int(batch.prefill_pages.shape[0] + batch.decode_pages.shape[0])
         self.ctx = B.Context(sh, batch.num_pages, max(batch.chunk_len, 1), max(batch.num_decode, 1),
                              total_pages + 16, device=device)
-        if prefill_rows is not None:
-            B.sw_debug_set_prefill_rows(self.ctx, prefill_rows)
         self.dbatch = B.DeviceBatch(batch, self.dev)
         self.pool = bits_to_torch(tensors["pool"], self.dev)
         self.q = bits_to_torch(tensors["q"], self.dev)

@@ -1,0 +1,71 @@
+"""The profiler (sw_cost_probe -> monotone table) and the serving loop on the GPU, at a size that takes seconds."""
+import numpy as np
+import pytest
+
+from paper_2609_07883_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def setup():
+    import torch
+
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_07883_b200 import build
+
+    build.build()
+    from paper_2609_07883_b200 import binding as B
+
+    shape, pages, layers = W.LLAMA, 4096, 2
+    dev = torch.device("cuda", 0)
+    ctx = B.Context(shape, pages, 512, 64, pages + 64)
+    pools = []
+    for layer in range(layers):
+        t = torch.zeros(pages * shape.page_elems, dtype=torch.bfloat16, device=dev)
+        W.fill_normal_bf16_(t, 900 + layer)
+        pools.append(t)
+    return B, ctx, pools, shape, pages
+
+
+def test_cost_probe_returns_ordered_percentiles(setup):
+    import torch
+
+    B, ctx, pools, shape, pages = setup
+    batch = W.make_batch(shape, pages, [700, 300, 1500], 256, 128, np.random.default_rng(1))
+    db = B.DeviceBatch(batch, pools[0].device)
+    q = torch.randn(batch.num_rows, shape.num_q_heads, shape.head_dim, device=pools[0].device).to(torch.bfloat16)
+    out = torch.empty_like(q)
+    p50, p99, samples = B.sw_cost_probe(ctx, pools, db, q, out, warmup=2, reps=20)
+    assert len(samples) == 20 and samples.min() > 0
+    assert samples.min() <= p50 <= p99 <= samples.max()
+    assert p50 == np.sort(samples)[9] and p99 == np.sort(samples)[19]   # nearest rank: ceil(q * reps)-th smallest
+    assert B.sw_check_status(ctx, raise_on_error=False) == (0, 0)
+
+
+def test_measured_table_is_made_monotone_and_drives_the_loop(setup):
+    B, ctx, pools, shape, pages = setup
+    from paper_2609_07883_b200 import profiler, serving
+
+    n_grid, ctx_grid, prefix_grid, chunk_grid = [1, 8, 64], [2048, 30000], [0, 4096], [0, 64, 256, 512]
+    tab = profiler.measure_table(ctx, pools, shape, pages, n_grid, ctx_grid, prefix_grid, chunk_grid, reps=4, warmup=1)
+    raw = np.asarray(tab["p99_ns"])
+    assert raw.shape == (3, 2, 2, 4) and (raw > 0).all()
+    table = profiler.to_cost_table(tab)
+    # the library's table is nondecreasing along every axis and never below the measurement
+    look = np.array([[[[table.lookup(n, c, p, k) for k in chunk_grid] for p in prefix_grid] for c in ctx_grid] for n in n_grid])
+    assert (look >= raw).all()
+    for ax in range(4):
+        assert (np.diff(look, axis=ax) >= 0).all()
+    # a short trace through the real executor: every admitted chunk must respect the quantum and the cap, and the
+    # device must report no problem
+    trace = W.bursty_trace(num_requests=24, rate_low=50.0, rate_high=200.0, mean_dwell_s=0.2, prompt_median=500.0,
+                           prompt_clip=(32, 3000), mean_output=12.0, rng=np.random.default_rng(3))
+    execute = serving.gpu_executor(ctx, pools, shape, 512, 64)
+    res = serving.run_trace(trace, 25.0, table, execute, shape, pages, policy="sloweave", c_max=512, max_decode=64,
+                            ctx_cap=ctx_grid[-1])
+    assert res["prefill_tokens"] == int(trace["prompt_len"].sum())
+    assert res["p99_chunk"] <= 512 and res["requests"] == 24
+    assert res["deadline_misses_with_chunk"] == 0
+    assert B.sw_check_status(ctx, raise_on_error=False) == (0, 0)
