@@ -340,6 +340,10 @@ __device__ __forceinline__ bool pf_mma(const MixedParams& p, const PfShared& sh,
 #ifndef SW_PF_SPLIT_MAX
 #define SW_PF_SPLIT_MAX 0
 #endif
+#ifndef SW_PF_MAX_CHAINS
+#define SW_PF_MAX_CHAINS 4
+#endif
+constexpr int kPfMaxChains = SW_PF_MAX_CHAINS;
 constexpr int kPolyEvery = SW_PF_POLY_EVERY;  // every kPolyEvery-th pair computes its first element with the polynomial; 0 = never
 template <bool kPoly>
 __device__ __forceinline__ float pf_exp2(float x) {
@@ -394,7 +398,6 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
         // the whole row of S (128 fp32) in registers: one TMEM read per element
         uint32_t s[128];
         const int limit = pos - j * 128 + 1;  // columns [0, limit) are attended
-        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x32(s_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
         tc_wait_ld();
@@ -402,14 +405,20 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
 #pragma unroll
             for (int i = 0; i < 128; ++i) s[i] = i < limit ? s[i] : 0xff800000u;  // -inf: exp2 gives exactly 0
         }
+        // row maximum: independent chains of 3-input max, then a short tree
+        float mxv[kPfMaxChains];
 #pragma unroll
-        for (int i = 0; i < 128; i += 8) {
-            mx0 = max3(mx0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
-            mx1 = max3(mx1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
-            mx2 = max3(mx2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
-            mx3 = max3(mx3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
-        }
-        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+        for (int c = 0; c < kPfMaxChains; ++c) mxv[c] = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 128; i += 2 * kPfMaxChains)
+#pragma unroll
+            for (int c = 0; c < kPfMaxChains; ++c)
+                mxv[c] = max3(mxv[c], __uint_as_float(s[i + 2 * c]), __uint_as_float(s[i + 2 * c + 1]));
+#pragma unroll
+        for (int w = kPfMaxChains / 2; w > 0; w >>= 1)
+#pragma unroll
+            for (int c = 0; c < w; ++c) mxv[c] = fmaxf(mxv[c], mxv[c + w]);
+        const float mx = mxv[0];
         const float m_new = fmaxf(m_ref, mx * sl2);
         if (j == it.j0) {
             m_ref = m_new;

@@ -223,3 +223,12 @@ def test_chat_workload_sampled_rows(gpu, oracle):
     prs = np.random.default_rng(5)
     pairs = [(r_, int(prs.integers(0, Hq))) for r_ in rows] + [(r_, int(prs.integers(0, Hq))) for r_ in rows]
     run_and_compare(gpu, oracle, batch, t, pairs=pairs, what="chat n=16 C=128")
+
+
+def test_many_decode_requests(gpu, oracle):
+    """1500 requests: the in-kernel plan scans several requests per thread and the unit search spans the whole list."""
+    rng = np.random.default_rng(40)
+    lens = rng.integers(1, 90, size=1500)
+    need = int(sum(-(-int(x) // 16) for x in lens)) + 8
+    batch = W.make_batch(W.TINY, need, lens, 0, 0, rng)
+    run_and_compare(gpu, oracle, batch, W.host_tensors(batch, rng), what="n=1500")

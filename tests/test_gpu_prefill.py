@@ -124,3 +124,12 @@ def test_dominant_key_and_constant_v_closed_forms(gpu, oracle):
     p = np.arange(257, dtype=np.float64)
     for h in range(8):
         assert np.max(np.abs(out2[:257, h, 0] - p / 512.0)) <= 4e-3
+
+
+@pytest.mark.parametrize("P,C", [(6000, 64), (20000, 32), (12000, 200)])
+def test_long_prefix_small_chunk_is_cut_into_pieces_and_merged(gpu, oracle, P, C):
+    """Few items with many KV tiles: each item is cut along the KV axis, published as partials and merged."""
+    rng = np.random.default_rng(P + C)
+    shape = W.AttnShape(8, 2, 128)
+    batch = W.make_batch(shape, (P + C) // 16 + 40, [300, 5], P, C, rng)
+    full_compare(gpu, oracle, batch, W.host_tensors(batch, rng), f"pieces P={P} C={C}")
