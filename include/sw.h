@@ -139,7 +139,8 @@ sw_status sw_decode_attn_static(const sw_layout* layout, int device, const void*
 
 /* Wait for `stream` and read the device status words: *code is 0 or the first device-detected problem as an
  * sw_status (bad page id / length → SW_ERR_OUT_OF_RANGE, bounded wait expired → SW_ERR_DEVICE_TIMEOUT),
- * *detail an implementation-defined locator.  The words are cleared.  Returns *code as status. */
+ * *detail an implementation-defined locator.  The words are cleared; after a reported problem the context's
+ * work counters and tickets are cleared too, so the next launch starts clean.  Returns *code as status. */
 sw_status sw_check_status(sw_ctx* ctx, void* stream, int32_t* code, int32_t* detail);
 
 /* ---- the controller (host only; no CUDA) ---------------------------------------------------------- */

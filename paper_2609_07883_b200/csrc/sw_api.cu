@@ -379,7 +379,10 @@ sw_status sw_check_status(sw_ctx* ctx, void* stream, int32_t* code, int32_t* det
     SW_CUDA(cudaMemcpyAsync(words, d, sizeof words, cudaMemcpyDeviceToHost, s));
     SW_CUDA(cudaStreamSynchronize(s));
     if (words[0] != 0) {
-        SW_CUDA(cudaMemsetAsync(d, 0, sizeof words, s));
+        // A launch that reported a problem may have skipped units or left early, so the work counters and tickets
+        // may not have been re-armed: clear them together with the status words (the stream is idle here).
+        SW_CUDA(cudaMemsetAsync(ctx->ws + ctx->w.ctrl, 0, ctx->w.part_ml - ctx->w.ctrl, s));
+        SW_CUDA(cudaMemsetAsync(ctx->ws + ctx->w.pf_tickets, 0, ctx->w.pf_ml - ctx->w.pf_tickets, s));
         SW_CUDA(cudaStreamSynchronize(s));
     }
     if (code) *code = words[0];

@@ -195,7 +195,7 @@ def main(argv=None):
     args = ap.parse_args(argv)
     build.build()
     rows = sweep(args.config, args.reps, lambda s: print(s, flush=True))
-    out = args.out or f"gpurun_out/cost_surface_{args.config}.json"
+    out = args.out or f"cost_surface_{args.config}.json"
     Path(out).parent.mkdir(parents=True, exist_ok=True)
     Path(out).write_text(json.dumps(rows, indent=1))
 

@@ -241,7 +241,7 @@ def main(argv=None):
     ap.add_argument("--margin-ppm", type=int, default=50_000)
     ap.add_argument("--table", default=None, help="JSON cost table to reuse; measured first when absent")
     ap.add_argument("--table-reps", type=int, default=8)
-    ap.add_argument("--out", default="gpurun_out/bursty.json")
+    ap.add_argument("--out", default="bursty_results.json")
     args = ap.parse_args(argv)
 
     build.build()

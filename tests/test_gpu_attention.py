@@ -232,3 +232,32 @@ def test_many_decode_requests(gpu, oracle):
     need = int(sum(-(-int(x) // 16) for x in lens)) + 8
     batch = W.make_batch(W.TINY, need, lens, 0, 0, rng)
     run_and_compare(gpu, oracle, batch, W.host_tensors(batch, rng), what="n=1500")
+
+
+def test_short_page_list_is_reported_and_the_context_recovers(gpu, oracle):
+    """A request whose page list is shorter than its length: its units are skipped and reported; reading the status
+    re-arms the context, and the next (good) iteration on the same context is correct."""
+    rng = np.random.default_rng(41)
+    shape = W.AttnShape(8, 2, 128)
+    lens = [5000, 3000]
+    need = sum(-(-x // 16) for x in lens) + 8
+    batch = W.make_batch(shape, need, lens, 0, 0, rng)
+    t = W.host_tensors(batch, rng)
+    r = gpu.Runner(batch, t)
+    B = r.B
+    bad = W.MixedBatch(**{**batch.__dict__})
+    bad.decode_page_indptr = batch.decode_page_indptr.copy()
+    bad.decode_page_indptr[1:] -= 100          # request 0 now owns 100 pages fewer than 5000 tokens need
+    bad.decode_pages = np.concatenate([batch.decode_pages[:batch.decode_page_indptr[1] - 100],
+                                       batch.decode_pages[batch.decode_page_indptr[1]:]])
+    B.sw_mixed_attn_run(r.ctx, r.pool, B.DeviceBatch(bad, r.dev), r.q, r.out)
+    code, _ = r.status()
+    assert code == B.SW_ERR_OUT_OF_RANGE
+    r.append()
+    r.attend()
+    out, lse = r.results()
+    assert r.status() == (0, 0)
+    pool = t["pool"].copy()
+    oracle.kv_append(pool, batch, t["k_new"], t["v_new"])
+    ref, ref_lse, _ = oracle.mixed_attention(pool, batch, t["q"])
+    gpu.compare(out.reshape(-1, 128), lse.reshape(-1), ref, ref_lse, "after recovery")
