@@ -143,6 +143,12 @@ sw_status sw_decode_attn_static(const sw_layout* layout, int device, const void*
  * work counters and tickets are cleared too, so the next launch starts clean.  Returns *code as status. */
 sw_status sw_check_status(sw_ctx* ctx, void* stream, int32_t* code, int32_t* detail);
 
+/* Self-test of the failure path (no counterpart in the paper): launches one warp that waits on a barrier nothing will
+ * ever complete.  Every device-side wait of this library is bounded; this one gives up after `budget_cycles` SM cycles
+ * (at most 4e9), records SW_ERR_DEVICE_TIMEOUT in the status words and ends normally — the context stays usable and
+ * sw_check_status then returns SW_ERR_DEVICE_TIMEOUT once.  Asynchronous on `stream`. */
+sw_status sw_selftest_wait_timeout(sw_ctx* ctx, int64_t budget_cycles, void* stream);
+
 /* ---- the controller (host only; no CUDA) ---------------------------------------------------------- */
 
 /* Cost table T^(n, ctx, prefix, c) in integer nanoseconds (Sec. 5.1: lookup table indexed by decode batch

@@ -50,7 +50,7 @@ class sw_choice(C.Structure):
 EXPORTS = ["sw_workspace_bytes", "sw_create", "sw_destroy", "sw_kv_append", "sw_mixed_attn_run",
            "sw_mixed_iteration_host", "sw_cost_probe", "sw_check_status", "sw_cost_table_create",
            "sw_cost_table_destroy", "sw_cost_table_lookup", "sw_choose_chunk", "sw_last_error",
-           "sw_decode_attn_static"]
+           "sw_decode_attn_static", "sw_selftest_wait_timeout"]
 
 _vp, _i32, _i64 = C.c_void_p, C.c_int32, C.c_int64
 _lib.sw_workspace_bytes.restype = C.c_size_t
@@ -64,6 +64,7 @@ _lib.sw_mixed_iteration_host.argtypes = [_vp, _vp, C.POINTER(sw_batch), _vp, _vp
 _lib.sw_cost_probe.argtypes = [_vp, C.POINTER(_vp), _i32, C.POINTER(sw_batch), _vp, _vp, _i32, _i32,
                                C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), _vp]
 _lib.sw_decode_attn_static.argtypes = [C.POINTER(sw_layout), C.c_int, _vp, C.POINTER(sw_batch), _vp, _vp, _vp, _vp]
+_lib.sw_selftest_wait_timeout.argtypes = [_vp, _i64, _vp]
 _lib.sw_check_status.argtypes = [_vp, _vp, C.POINTER(_i32), C.POINTER(_i32)]
 _lib.sw_cost_table_create.argtypes = [C.POINTER(_i32), _i32, C.POINTER(_i64), _i32, C.POINTER(_i32), _i32,
                                       C.POINTER(_i32), _i32, C.POINTER(_i64), C.c_int, C.c_int, C.POINTER(_vp)]
@@ -211,6 +212,11 @@ def sw_check_status(ctx: Context, stream=None, raise_on_error: bool = True):
 
 
 SW_STATIC_MAX_DECODE = 128
+
+
+def sw_selftest_wait_timeout(ctx: Context, budget_cycles: int = 200_000, stream=None) -> None:
+    """Launch the bounded-wait self-test: a wait that cannot succeed gives up and reports SW_ERR_DEVICE_TIMEOUT."""
+    _check(_lib.sw_selftest_wait_timeout(ctx.handle, int(budget_cycles), _stream_handle(stream)), "sw_selftest_wait_timeout")
 
 
 def sw_decode_attn_static(layout: sw_layout, device: int, kv_pool, batch: DeviceBatch, q, out, lse=None, stream=None) -> None:

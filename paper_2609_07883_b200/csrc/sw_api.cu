@@ -393,4 +393,12 @@ sw_status sw_check_status(sw_ctx* ctx, void* stream, int32_t* code, int32_t* det
     return SW_OK;
 }
 
+sw_status sw_selftest_wait_timeout(sw_ctx* ctx, int64_t budget_cycles, void* stream) {
+    if (!ctx || budget_cycles < 0 || budget_cycles > 4000000000LL)
+        return sw_fail(SW_ERR_INVALID_ARG, "sw_selftest_wait_timeout: invalid argument (budget of at most 4e9 cycles)");
+    SW_CUDA(sw::launch_selftest_wait(reinterpret_cast<int32_t*>(ctx->ws + ctx->w.ctrl), (long long)budget_cycles,
+                                     static_cast<cudaStream_t>(stream)));
+    return SW_OK;
+}
+
 }  // extern "C"

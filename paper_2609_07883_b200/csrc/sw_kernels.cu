@@ -599,6 +599,24 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     }
 }
 
+// Self-test of the bounded wait: one warp waits on a barrier that nothing will ever complete; the wait must give up
+// after `budget_cycles`, record SW_ERR_DEVICE_TIMEOUT in the status word and let the kernel end normally.
+__global__ void sw_selftest_wait_kernel(int32_t* ctrl, long long budget_cycles) {
+    __shared__ __align__(8) unsigned long long bar;
+    const uint32_t addr = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(addr, 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+    if (!mbar_wait(addr, 0, budget_cycles) && threadIdx.x == 0) report(ctrl, SW_ERR_DEVICE_TIMEOUT, kSiteWait, 0xABCD);
+}
+
+cudaError_t launch_selftest_wait(int32_t* ctrl, long long budget_cycles, cudaStream_t stream) {
+    sw_selftest_wait_kernel<<<1, 32, 0, stream>>>(ctrl, budget_cycles);
+    return cudaGetLastError();
+}
+
 size_t mixed_attn_smem_bytes(int head_dim) {
     return (head_dim == 64 ? Geo<64>::kSmemBytes : Geo<128>::kSmemBytes) + 1024;
 }

@@ -261,3 +261,21 @@ def test_short_page_list_is_reported_and_the_context_recovers(gpu, oracle):
     oracle.kv_append(pool, batch, t["k_new"], t["v_new"])
     ref, ref_lse, _ = oracle.mixed_attention(pool, batch, t["q"])
     gpu.compare(out.reshape(-1, 128), lse.reshape(-1), ref, ref_lse, "after recovery")
+
+
+def test_a_wait_that_cannot_succeed_gives_up_and_the_context_stays_usable(gpu, oracle):
+    """Failure detection without a fault: a bounded wait runs out (nothing ever completes its barrier), the kernel ends
+    normally with SW_ERR_DEVICE_TIMEOUT in the status word, and the same context then runs a correct iteration."""
+    import time
+
+    rng = np.random.default_rng(42)
+    batch = W.make_batch(W.TINY, 64, [40, 70], 10, 20, rng)
+    t = W.host_tensors(batch, rng)
+    r = gpu.Runner(batch, t)
+    t0 = time.time()
+    r.B.sw_selftest_wait_timeout(r.ctx, 200_000)          # about 0.1 ms of SM clock
+    code, detail = r.status()
+    assert time.time() - t0 < 5.0
+    assert code == r.B.SW_ERR_DEVICE_TIMEOUT and (detail & 0xFFFFFF) == 0xABCD
+    assert r.status() == (0, 0)
+    run_and_compare(gpu, oracle, batch, t, what="after a timed-out wait")
