@@ -16,9 +16,7 @@
 
 namespace {
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+using sw::EncodeTiledFn;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -76,7 +74,7 @@ struct sw_ctx {
     EncodeTiledFn encode = nullptr;
     struct MapEntry {
         const void* pool;
-        CUtensorMap map;
+        sw::KvMaps maps;
     };
     std::vector<MapEntry> kv_maps;  // small cache: one entry per pool of a layer stack
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -90,30 +88,21 @@ namespace {
         if (e_ != cudaSuccess) return sw_fail(SW_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_));  \
     } while (0)
 
-sw_status kv_map_for(sw_ctx* ctx, const void* pool, const CUtensorMap** out) {
+sw_status kv_map_for(sw_ctx* ctx, const void* pool, const sw::KvMaps** out) {
     for (auto& e : ctx->kv_maps)
         if (e.pool == pool) {
-            *out = &e.map;
+            *out = &e.maps;
             return SW_OK;
         }
     const sw_layout& l = ctx->layout;
     if ((reinterpret_cast<uintptr_t>(pool) & 15) != 0) return sw_fail(SW_ERR_INVALID_ARG, "kv_pool must be 16-byte aligned");
-    // [page][K|V x kv head][slot][element]; one box = [16 slots][64 elements] = one 128-byte-swizzled block
-    const cuuint64_t dims[4] = {(cuuint64_t)l.head_dim, (cuuint64_t)sw::kPageSize, (cuuint64_t)2 * l.num_kv_heads,
-                                (cuuint64_t)l.num_pages};
-    const cuuint64_t strides[3] = {(cuuint64_t)l.head_dim * 2, (cuuint64_t)sw::kPageSize * l.head_dim * 2,
-                                   (cuuint64_t)2 * l.num_kv_heads * sw::kPageSize * l.head_dim * 2};
-    const cuuint32_t box[4] = {64, (cuuint32_t)sw::kPageSize, 1, 1};
-    const cuuint32_t elem_strides[4] = {1, 1, 1, 1};
     sw_ctx::MapEntry e;
     e.pool = pool;
-    CUresult r = ctx->encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), dims, strides, box,
-                             elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = sw::encode_kv_maps(ctx->encode, l, pool, &e.maps);
     if (r != CUDA_SUCCESS) return sw_fail(SW_ERR_CUDA, "cuTensorMapEncodeTiled(kv pool) failed with CUresult %d", (int)r);
     if (ctx->kv_maps.size() >= 128) ctx->kv_maps.erase(ctx->kv_maps.begin());
     ctx->kv_maps.push_back(e);
-    *out = &ctx->kv_maps.back().map;
+    *out = &ctx->kv_maps.back().maps;
     return SW_OK;
 }
 
@@ -239,8 +228,8 @@ sw_status sw_mixed_attn_run(sw_ctx* ctx, const void* kv_pool, const sw_batch* ba
     if (!kv_pool || !q || !out) return sw_fail(SW_ERR_INVALID_ARG, "sw_mixed_attn_run: null tensor");
     if (((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) & 15) != 0)
         return sw_fail(SW_ERR_INVALID_ARG, "sw_mixed_attn_run: q and out must be 16-byte aligned");
-    const CUtensorMap* kv_map = nullptr;
-    st = kv_map_for(ctx, kv_pool, &kv_map);
+    const sw::KvMaps* kv_maps = nullptr;
+    st = kv_map_for(ctx, kv_pool, &kv_maps);
     if (st != SW_OK) return st;
     const sw_layout& l = ctx->layout;
     sw::MixedParams p{};
@@ -272,7 +261,7 @@ sw_status sw_mixed_attn_run(sw_ctx* ctx, const void* kv_pool, const sw_batch* ba
     p.pf_tickets = reinterpret_cast<int32_t*>(ctx->ws + ctx->w.pf_tickets);
     // q as [row][head][element] restricted to the chunk rows: one box = 128 tile rows (token-major, the g heads of a
     // KV head minor) x 64 elements; rows past the chunk read as zero
-    CUtensorMap q_map = *kv_map;
+    CUtensorMap q_map = kv_maps->tile;
     if (p.C > 0) {
         const cuuint64_t dims[3] = {(cuuint64_t)l.head_dim, (cuuint64_t)l.num_q_heads, (cuuint64_t)p.C};
         const cuuint64_t strides[2] = {(cuuint64_t)l.head_dim * 2, (cuuint64_t)l.num_q_heads * l.head_dim * 2};
@@ -283,7 +272,7 @@ sw_status sw_mixed_attn_run(sw_ctx* ctx, const void* kv_pool, const sw_batch* ba
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return sw_fail(SW_ERR_CUDA, "cuTensorMapEncodeTiled(q) failed with CUresult %d", (int)r);
     }
-    SW_CUDA(sw::launch_mixed_attn(l.head_dim, *kv_map, q_map, p, ctx->num_sms, static_cast<cudaStream_t>(stream)));
+    SW_CUDA(sw::launch_mixed_attn(l.head_dim, *kv_maps, q_map, p, ctx->num_sms, static_cast<cudaStream_t>(stream)));
     return SW_OK;
 }
 

@@ -70,9 +70,45 @@ struct AppendParams {
     int32_t* ctrl;
 };
 
+// Tensor maps of one KV pool [page][K|V][kv head][slot][element].
+//   tile: 4-D {element, slot, K|V x kv head, page}, box = [16 slots][64 elements], one 128-byte-swizzled block; the
+//         chunk-prefill producer lays such blocks out as 128-key MMA operand tiles.
+//   page: 5-D {element % 64, slot, element / 64, 2 * page + K|V, kv head}, box = all of one head's K and V in a page
+//         (2 x head_dim/64 blocks of the same swizzled form, K blocks first): a decode unit fetches a page with one copy.
+struct KvMaps {
+    CUtensorMap tile;
+    CUtensorMap page;
+};
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+inline CUresult encode_kv_maps(EncodeTiledFn encode, const sw_layout& l, const void* pool, KvMaps* out) {
+    const cuuint64_t row = (cuuint64_t)l.head_dim * 2;                 // bytes of one slot of one head
+    const cuuint64_t head = (cuuint64_t)kPageSize * row;               // one head's K (or V) in a page
+    const cuuint64_t side = (cuuint64_t)l.num_kv_heads * head;         // all K (or all V) of a page
+    const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+    {
+        const cuuint64_t dims[4] = {(cuuint64_t)l.head_dim, (cuuint64_t)kPageSize, (cuuint64_t)2 * l.num_kv_heads,
+                                    (cuuint64_t)l.num_pages};
+        const cuuint64_t strides[3] = {row, head, 2 * side};
+        const cuuint32_t box[4] = {64, (cuuint32_t)kPageSize, 1, 1};
+        CUresult r = encode(&out->tile, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), dims, strides, box, ones,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return r;
+    }
+    const cuuint64_t dims[5] = {64, (cuuint64_t)kPageSize, (cuuint64_t)l.head_dim / 64, (cuuint64_t)2 * l.num_pages,
+                                (cuuint64_t)l.num_kv_heads};
+    const cuuint64_t strides[4] = {row, 128, side, head};
+    const cuuint32_t box[5] = {64, (cuuint32_t)kPageSize, (cuuint32_t)l.head_dim / 64, 2, 1};
+    return encode(&out->page, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(pool), dims, strides, box, ones,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
 // launchers (sw_kernels.cu)
 cudaError_t launch_kv_append(const AppendParams& p, cudaStream_t stream);
-cudaError_t launch_mixed_attn(int head_dim, const CUtensorMap& kv_map, const CUtensorMap& q_map, const MixedParams& p,
+cudaError_t launch_mixed_attn(int head_dim, const KvMaps& kv_maps, const CUtensorMap& q_map, const MixedParams& p,
                               int num_sms, cudaStream_t stream);
 cudaError_t configure_kernels(int head_dim);
 cudaError_t launch_selftest_wait(int32_t* ctrl, long long budget_cycles, cudaStream_t stream);

@@ -110,17 +110,23 @@ struct Geo {
     static constexpr int kBarOffset = kRingBytes;                              // kWarps*kStages mbarriers
     static constexpr int kPfBarOffset = kBarOffset + kWarps * kStages * 8;     // barriers of the prefill tiles
     static constexpr int kPlanOffset = kPfBarOffset + 32 * 8;                  // int32 unit_prefix[kMaxDecode+1]
-    static constexpr int kMiscOffset = kPlanOffset + (kMaxDecode + 1) * 4 + 12; // scan scratch, TMEM base, abort flag
-    static constexpr int kSmemBytes = kMiscOffset + 256;
+    static constexpr int kLenOffset = kPlanOffset + (kMaxDecode + 1) * 4 + 12;  // int32 kv_len[kMaxDecode]
+    static constexpr int kIndptrOffset = kLenOffset + kMaxDecode * 4;           // int32 page_indptr[kMaxDecode+1]
+    static constexpr int kMiscOffset = kIndptrOffset + (kMaxDecode + 1) * 4 + 12; // scan scratch, TMEM base, abort flag
+    static constexpr int kSmemBytes = kMiscOffset + 512;   // 64 ints scan scratch and flags, then the plan's counter
 };
 
+constexpr int kOneRoundMaxPages = 48;  // longest unit (pages) for which one round of units is planned
 struct Plan {
+    const int* len;     // shared-memory copies of the context lengths and page-list offsets
+    const int* indptr;
     int split_tokens;   // tokens per split-KV unit (multiple of the page size)
     int decode_units;   // sum over requests of ceil(len / split_tokens)
     int total_items;
 };
 
-// Block-wide exclusive scan of one value per thread (kThreads threads).  scratch: kWarps+1 ints.
+// Block-wide exclusive scan of one value per thread (kThreads threads): a warp scan, one barrier, then every thread
+// adds up the warps before its own.  scratch: kWarps ints nobody has touched since the last barrier; one use only.
 __device__ __forceinline__ int block_exclusive_scan(int v, int* scratch, int* total) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int inc = v;
@@ -131,27 +137,31 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* scratch, int* to
     }
     if (lane == 31) scratch[warp] = inc;
     __syncthreads();
-    if (warp == 0) {
-        int w = lane < kWarps ? scratch[lane] : 0;
-        int winc = w;
+    int before = 0, all = 0;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int t = __shfl_up_sync(0xffffffffu, winc, o);
-            if (lane >= o) winc += t;
-        }
-        if (lane < kWarps) scratch[lane] = winc - w;
-        if (lane == kWarps - 1) scratch[kWarps] = winc;
+    for (int w = 0; w < kWarps; ++w) {
+        const int t = scratch[w];
+        all += t;
+        if (w < warp) before += t;
     }
+    *total = all;
+    return before + inc - v;
+}
+
+// Block-wide sum of one value per thread: a warp reduction, one shared-memory add per warp, one barrier.  ctr is a
+// counter that was zero before the previous barrier; one use only.
+__device__ __forceinline__ int block_sum(int v, int* ctr) {
+    const int w = __reduce_add_sync(0xffffffffu, v);
+    if ((threadIdx.x & 31) == 0 && w != 0) atomicAdd(ctr, w);
     __syncthreads();
-    const int r = scratch[warp] + inc - v;
-    *total = scratch[kWarps];
-    __syncthreads();
-    return r;
+    return *reinterpret_cast<volatile int*>(ctr);
 }
 
 // Every CTA derives the same plan from the context lengths: no host planning, no extra launch.
-__device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix, int* scratch) {
+__device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix, int* len_s, int* indptr_s, int* scratch) {
     Plan plan;
+    plan.len = len_s;
+    plan.indptr = indptr_s;
     const int per_thread = (p.n + kThreads - 1) / kThreads;
     const int beg = min(p.n, (int)threadIdx.x * per_thread);
     const int end = min(p.n, beg + per_thread);
@@ -160,17 +170,17 @@ __device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix
     for (int i = beg; i < end; ++i) {
         const int len = p.decode_kv_len[i];
         pages_local += len > 0 ? (len + kPageSize - 1) / kPageSize : 0;
-        // the units read these offsets later: bring their lines into L1 now
-        asm volatile("prefetch.global.L1 [%0];" ::"l"(p.decode_page_indptr + i));
+        len_s[i] = len;                              // the units read these from shared memory later
+        indptr_s[i] = p.decode_page_indptr[i];
     }
-    int total_pages = 0;
-    block_exclusive_scan(pages_local, scratch, &total_pages);
+    if (threadIdx.x == 0 && p.n > 0) indptr_s[p.n] = p.decode_page_indptr[p.n];
+    const int total_pages = block_sum(pages_local, scratch + 64);  // counter zeroed in the kernel prologue
     // Unit size.  Small batches are latency-bound: one round of units, as many as there are warps, gets every warp
     // streaming at once.  Large batches are bandwidth-bound: a few rounds of smaller units shorten the tail.  Every
     // request adds at most one ragged unit per head, hence the "- n".
     const int per_head_warps = max(1, (int)gridDim.x * kWarps / p.Hkv);
     const int one_round = (total_pages + per_head_warps - 1) / per_head_warps;  // pages per unit if run in one round
-    const int rounds = one_round <= 48 ? 1 : (one_round <= 160 ? 2 : 4);
+    const int rounds = one_round <= kOneRoundMaxPages ? 1 : (one_round <= 160 ? 2 : 4);
     int units_target = max(1, rounds * per_head_warps - p.n);
     units_target = min(units_target, max(1, p.target_items / p.Hkv));
     int split_pages = (total_pages + units_target - 1) / units_target;
@@ -178,14 +188,14 @@ __device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix
     plan.split_tokens = split_pages * kPageSize;
     int units_local = 0;
     for (int i = beg; i < end; ++i) {
-        const int len = p.decode_kv_len[i];
+        const int len = len_s[i];
         units_local += len > 0 ? (len + plan.split_tokens - 1) / plan.split_tokens : 0;
     }
     int total_units = 0;
     int run = block_exclusive_scan(units_local, scratch, &total_units);
     for (int i = beg; i < end; ++i) {
         unit_prefix[i] = run;
-        const int len = p.decode_kv_len[i];
+        const int len = len_s[i];
         run += len > 0 ? (len + plan.split_tokens - 1) / plan.split_tokens : 0;
     }
     if (threadIdx.x == 0) unit_prefix[p.n] = total_units;
@@ -217,25 +227,141 @@ struct WarpRing {
     uint32_t it;    // pages consumed so far (stage = it % kStages, parity = (it / kStages) & 1)
 };
 
-// Whole-warp call: lane 0 arms the stage's barrier, lanes 0 .. 2*halves-1 each issue one of the page's boxes.
+// Lane 0 arms the stage's barrier and fetches the page with one copy: the head's K blocks, then its V blocks.
 template <int D>
-__device__ __forceinline__ void issue_page(const CUtensorMap* kv_map, const WarpRing<D>& ring, uint32_t issue_it, int page,
-                                           int kvh, int Hkv) {
+__device__ __forceinline__ void issue_page(const CUtensorMap* kvp_map, const WarpRing<D>& ring, uint32_t issue_it, int page,
+                                           int kvh) {
+    if ((threadIdx.x & 31) == 0) {
+        const uint32_t stage = issue_it % kStages;
+        const uint32_t bar = ring.bar + stage * 8;
+        mbar_arrive_expect_tx(bar, Geo<D>::kStageBytes);
+        tma_load_5d(ring.buf + stage * Geo<D>::kStageBytes, kvp_map, bar, 0, 0, 0, 2 * page, kvh);
+    }
+}
+
+// Merge of the splits of one (request, kv head) by the last unit to arrive, all rows together so that the loads of
+// one pass are in flight at once.  G >= group size is a compile-time bound: rows beyond the group read row 0 with
+// weight zero, which keeps the loops free of branches.  Slots of the splits are Hkv apart.
+template <int D, int G>
+__device__ __forceinline__ void merge_splits(const MixedParams& p, const Unit& u) {
+    constexpr int V = D / 32;                 // output columns per lane
+    constexpr int J = G >= 8 ? 2 : (G == 4 ? 4 : 8);  // splits whose partial outputs are loaded together
     const int lane = threadIdx.x & 31;
-    const uint32_t stage = issue_it % kStages;
-    const uint32_t dst = ring.buf + stage * Geo<D>::kStageBytes;
-    const uint32_t bar = ring.bar + stage * 8;
-    if (lane == 0) mbar_arrive_expect_tx(bar, Geo<D>::kStageBytes);
-    __syncwarp();
-    if (lane < 2 * Geo<D>::kHalves) {
-        const int x = lane / Geo<D>::kHalves, h = lane % Geo<D>::kHalves;
-        tma_load_4d(dst + lane * Geo<D>::kBlockBytes, kv_map, bar, h * 64, 0, x * Hkv + kvh, page);
+    const int g = p.group;
+    const int slot0 = u.slot - u.split * p.Hkv;
+    const int ns = u.nsplit;
+    const float* ml0 = p.part_ml + (int64_t)slot0 * (2 * kMaxGroup);  // split s: + s * ml_stride
+    const int64_t ml_stride = (int64_t)p.Hkv * (2 * kMaxGroup);
+    // pass 1: lanes take splits; per row the running maximum and the row sum rescaled to it, then one warp reduction
+    float m_all[G], l_all[G], m_first[G];
+#pragma unroll
+    for (int r = 0; r < G; ++r) {
+        m_all[r] = -INFINITY;
+        l_all[r] = 0.f;
+        m_first[r] = -INFINITY;
+    }
+    for (int s0 = 0; s0 < ns; s0 += 32) {
+        const int sidx = min(s0 + lane, ns - 1);
+        const bool live = s0 + lane < ns;
+        float ms[G], ls[G];
+#pragma unroll
+        for (int r = 0; r < G; ++r) {
+            const int rr = r < g ? r : 0;
+            ms[r] = __ldcg(ml0 + sidx * ml_stride + rr);
+            ls[r] = __ldcg(ml0 + sidx * ml_stride + kMaxGroup + rr);
+        }
+#pragma unroll
+        for (int r = 0; r < G; ++r) {
+            if (!live) ms[r] = -INFINITY;
+            if (s0 == 0) m_first[r] = ms[r];
+            const float m_new = fmaxf(m_all[r], ms[r]);
+            const float a = m_all[r] == -INFINITY ? 0.f : fast_exp2((m_all[r] - m_new) * p.sm_scale_log2);
+            const float b = ms[r] == -INFINITY ? 0.f : fast_exp2((ms[r] - m_new) * p.sm_scale_log2);
+            l_all[r] = l_all[r] * a + ls[r] * b;
+            m_all[r] = m_new;
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < G; ++r) {
+        float mw = m_all[r];
+#pragma unroll
+        for (int o2 = 16; o2 > 0; o2 >>= 1) mw = fmaxf(mw, __shfl_xor_sync(0xffffffffu, mw, o2));
+        float lw = m_all[r] == -INFINITY ? 0.f : l_all[r] * fast_exp2((m_all[r] - mw) * p.sm_scale_log2);
+#pragma unroll
+        for (int o2 = 16; o2 > 0; o2 >>= 1) lw += __shfl_xor_sync(0xffffffffu, lw, o2);
+        m_all[r] = mw;
+        l_all[r] = lw;
+    }
+    // pass 2: weighted sum of the partial outputs; lanes take V adjacent columns of every row, J splits per batch
+    float acc[G][V];
+#pragma unroll
+    for (int r = 0; r < G; ++r)
+#pragma unroll
+        for (int v = 0; v < V; ++v) acc[r][v] = 0.f;
+    const float* po0 = p.part_o + (int64_t)slot0 * g * D + lane * V;  // split s, row r: + s * po_stride + r * D
+    const int64_t po_stride = (int64_t)p.Hkv * g * D;
+    for (int s0 = 0; s0 < ns; s0 += 32) {
+        float w[G];
+#pragma unroll
+        for (int r = 0; r < G; ++r) {
+            float ms = m_first[r];
+            if (s0 > 0) {
+                ms = __ldcg(ml0 + min(s0 + lane, ns - 1) * ml_stride + (r < g ? r : 0));
+                if (s0 + lane >= ns) ms = -INFINITY;
+            }
+            w[r] = (ms == -INFINITY || r >= g) ? 0.f : fast_exp2((ms - m_all[r]) * p.sm_scale_log2);
+        }
+        const int cnt = min(32, ns - s0);
+        for (int j0 = 0; j0 < cnt; j0 += J) {
+            float x[J][G][V];
+#pragma unroll
+            for (int j = 0; j < J; ++j) {
+                const float* src = po0 + (s0 + min(j0 + j, cnt - 1)) * po_stride;
+#pragma unroll
+                for (int r = 0; r < G; ++r) {
+                    const float* row = src + (r < g ? r : 0) * D;
+                    if constexpr (V == 4) {
+                        const float4 t = __ldcg(reinterpret_cast<const float4*>(row));
+                        x[j][r][0] = t.x, x[j][r][1] = t.y, x[j][r][2] = t.z, x[j][r][3] = t.w;
+                    } else {
+                        const float2 t = __ldcg(reinterpret_cast<const float2*>(row));
+                        x[j][r][0] = t.x, x[j][r][1] = t.y;
+                    }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < J; ++j) {
+#pragma unroll
+                for (int r = 0; r < G; ++r) {
+                    float wj = __shfl_sync(0xffffffffu, w[r], (j0 + j) & 31);
+                    if (j0 + j >= cnt) wj = 0.f;
+#pragma unroll
+                    for (int v = 0; v < V; ++v) acc[r][v] = fmaf(wj, x[j][r][v], acc[r][v]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < G; ++r) {
+        if (r < g) {
+            const float inv = 1.f / l_all[r];
+            const int hd = u.kvh * g + r;
+            __nv_bfloat16* dst = p.out + ((int64_t)u.q_row * p.Hq + hd) * D + lane * V;
+            if constexpr (V == 4) {
+                *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16x2(acc[r][0] * inv, acc[r][1] * inv),
+                                                            pack_bf16x2(acc[r][2] * inv, acc[r][3] * inv));
+            } else {
+                *reinterpret_cast<uint32_t*>(dst) = pack_bf16x2(acc[r][0] * inv, acc[r][1] * inv);
+            }
+            if (p.lse && lane == 0) p.lse[(int64_t)u.q_row * p.Hq + hd] = m_all[r] * p.sm_scale + __logf(l_all[r]);
+        }
     }
 }
 
 // Runs one unit; returns false if a bounded wait expired.
 template <int D>
-__device__ bool run_unit(const CUtensorMap* kv_map, const MixedParams& p, const Unit& u, WarpRing<D>& ring) {
+__device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const Unit& u, WarpRing<D>& ring, int fixed_items,
+                         int& next_item) {
     constexpr int KS = D / 16;  // k-slices of QK^T; also pairs of 8-wide output column tiles of PV
     const int lane = threadIdx.x & 31;
     const int qrow_in_group = lane >> 2;  // accumulator row held in c0/c1
@@ -286,10 +412,20 @@ __device__ bool run_unit(const CUtensorMap* kv_map, const MixedParams& p, const 
         if (page < 0 || (int64_t)page >= p.num_pages) {
             if (lane == 0) report(p.ctrl, SW_ERR_OUT_OF_RANGE, kSiteAttnPage, u.q_row);
         }
-        issue_page<D>(kv_map, ring, it0 + issued, page, u.kvh, p.Hkv);
+        issue_page<D>(kvp_map, ring, it0 + issued, page, u.kvh);
         ++issued;
     };
     for (int k = 0; k < kStages && k < npg; ++k) issue_next();
+    // Once this unit's last page is on its way the following unit is claimed from the shared counter: the counter's
+    // round trip hides behind the last pages, and no warp hoards a unit while others are still idle.
+    bool claimed = false;
+    auto claim_next = [&]() {
+        if (!claimed && issued >= npg) {
+            claimed = true;
+            if (lane == 0) next_item = fixed_items + atomicAdd(&p.ctrl[kCtrWork], 1);
+        }
+    };
+    claim_next();
 
     for (int k = 0; k < npg; ++k) {
         const uint32_t stage = ring.it % kStages;
@@ -386,6 +522,7 @@ __device__ bool run_unit(const CUtensorMap* kv_map, const MixedParams& p, const 
         __syncwarp();  // every lane is done reading this stage before it is refilled
         if (valid_hi < kPageSize) fence_proxy_async_smem();
         if (issued < npg) issue_next();
+        claim_next();
     }
 
     // finish: row sums across the quad
@@ -422,45 +559,14 @@ __device__ bool run_unit(const CUtensorMap* kv_map, const MixedParams& p, const 
     prev = __shfl_sync(0xffffffffu, prev, 0);
     if (prev != u.nsplit - 1) return true;
 
-    // last arriver: merge all splits of this (request, kv head); slots of its splits are Hkv apart
+    // last arriver: merge all splits of this (request, kv head)
     __threadfence();
     if (lane == 0) p.tickets[u.ticket] = 0;  // ready for the next launch
-    const int slot0 = u.slot - u.split * p.Hkv;
-    const int ns = u.nsplit;
-    for (int r = 0; r < g; ++r) {
-        // running maximum and weighted sum over the splits: lanes take splits, then one warp reduction each
-        const float* ml = p.part_ml + (int64_t)slot0 * (2 * kMaxGroup) + r;   // split s: + s * ml_stride
-        const int64_t ml_stride = (int64_t)p.Hkv * (2 * kMaxGroup);
-        float m_all = -INFINITY;
-        for (int sidx = lane; sidx < ns; sidx += 32) m_all = fmaxf(m_all, __ldcg(ml + sidx * ml_stride));
-#pragma unroll
-        for (int o2 = 16; o2 > 0; o2 >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xffffffffu, m_all, o2));
-        float l_all = 0.f;
-        for (int sidx = lane; sidx < ns; sidx += 32) {
-            const float ms = __ldcg(ml + sidx * ml_stride);
-            l_all += (ms == -INFINITY ? 0.f : fast_exp2((ms - m_all) * p.sm_scale_log2)) * __ldcg(ml + sidx * ml_stride + kMaxGroup);
-        }
-#pragma unroll
-        for (int o2 = 16; o2 > 0; o2 >>= 1) l_all += __shfl_xor_sync(0xffffffffu, l_all, o2);
-        // weighted sum of the partial outputs: lanes take columns, eight splits' loads in flight
-        float acc[D / 32];
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) acc[c] = 0.f;
-        const float* po = p.part_o + ((int64_t)slot0 * g + r) * D + lane;      // split s: + s * po_stride
-        const int64_t po_stride = (int64_t)p.Hkv * g * D;
-#pragma unroll 8
-        for (int sidx = 0; sidx < ns; ++sidx) {
-            const float ms = __ldcg(ml + sidx * ml_stride);
-            const float w = ms == -INFINITY ? 0.f : fast_exp2((ms - m_all) * p.sm_scale_log2);
-#pragma unroll
-            for (int c = 0; c < D / 32; ++c) acc[c] = fmaf(w, __ldcg(po + sidx * po_stride + c * 32), acc[c]);
-        }
-        const float inv = 1.f / l_all;
-        const int hd = u.kvh * g + r;
-        __nv_bfloat16* dst = p.out + ((int64_t)u.q_row * p.Hq + hd) * D;
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) dst[c * 32 + lane] = __float2bfloat16(acc[c] * inv);
-        if (p.lse && lane == 0) p.lse[(int64_t)u.q_row * p.Hq + hd] = m_all * p.sm_scale + __logf(l_all);
+    switch (g) {
+        case 1: merge_splits<D, 1>(p, u); break;
+        case 2: merge_splits<D, 2>(p, u); break;
+        case 4: merge_splits<D, 4>(p, u); break;
+        default: merge_splits<D, kMaxGroup>(p, u); break;
     }
     return true;
 }
@@ -474,6 +580,7 @@ namespace sw {
 // ---------------------------------------------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid_constant__ CUtensorMap kv_map,
+                                                                       const __grid_constant__ CUtensorMap kvp_map,
                                                                     const __grid_constant__ CUtensorMap q_map,
                                                                     const MixedParams p) {
     static_assert(PfGeo<D>::kBytes <= Geo<D>::kRingBytes, "prefill tiles must fit the region shared with the decode ring");
@@ -488,8 +595,10 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
 
     const bool tensor_prefill = p.C > 0;
     volatile int* misc = reinterpret_cast<volatile int*>(scratch + 32);  // [0] TMEM base, [1] abort flag, [2..3] ticket flags
+    if (threadIdx.x == 32) scratch[64] = 0;  // the plan's block-sum counter
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&kv_map);
+        tma_prefetch_desc(&kvp_map);
         for (int i = 0; i < kWarps * kStages; ++i) mbar_init(base + Geo<D>::kBarOffset + i * 8, 1);
         if (tensor_prefill) {
             tma_prefetch_desc(&q_map);
@@ -506,11 +615,13 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     __syncthreads();
 
     // chunk-prefill tiles first (long, tensor-bound); the decode units below fill the tail
+    // The first prefill entry of a CTA is its own index and the first decode unit of a warp is fixed as well: neither
+    // waits for a counter.  CTAs that start with prefill work take all their decode units from the counter.
+    int prefill_ctas = 0;
     if (tensor_prefill) {
         const PfPlan pplan = pf_make_plan(p);
-        if (threadIdx.x == 0) misc[4] = atomicAdd(&p.ctrl[kCtrPrefill], 1);
-        __syncthreads();
-        const int first_entry = misc[4];
+        prefill_ctas = min(pplan.n_entries, (int)gridDim.x);
+        const int first_entry = blockIdx.x;
         if (first_entry < pplan.n_entries) {  // CTA-uniform: this CTA has prefill work
             if (warp == 1) {
                 tmem_alloc(smem_u32(const_cast<int*>(&misc[0])), 512);
@@ -537,7 +648,8 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
         __syncthreads();
     }
 
-    const Plan plan = make_plan(p, unit_prefix, scratch);
+    const Plan plan = make_plan(p, unit_prefix, reinterpret_cast<int*>(smem + Geo<D>::kLenOffset),
+                                reinterpret_cast<int*>(smem + Geo<D>::kIndptrOffset), scratch);
     if (plan.total_items > p.max_items) {
         if (threadIdx.x == 0) report(p.ctrl, SW_ERR_WORKSPACE, kSiteScratch, plan.total_items);
     } else {
@@ -545,11 +657,14 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
         ring.buf = base + warp * kStages * Geo<D>::kStageBytes;
         ring.bar = base + Geo<D>::kBarOffset + warp * kStages * 8;
         ring.it = 0;
-        while (true) {
-            int item = 0;
-            if (lane == 0) item = atomicAdd(&p.ctrl[kCtrWork], 1);
+        const int fixed_items = ((int)gridDim.x - prefill_ctas) * kWarps;  // units handed out without the counter
+        int item = ((int)blockIdx.x - prefill_ctas) * kWarps + warp;
+        if ((int)blockIdx.x < prefill_ctas) {
+            if (lane == 0) item = fixed_items + atomicAdd(&p.ctrl[kCtrWork], 1);
             item = __shfl_sync(0xffffffffu, item, 0);
-            if (item >= plan.total_items) break;
+        }
+        while (item < plan.total_items) {
+            int next_item = 0;  // lane 0: claimed inside run_unit
             Unit u;
             bool ok = true;
             {
@@ -563,7 +678,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
                 }
                 const int i = lo;
                 u.q_row = p.C + i;
-                u.len = p.decode_kv_len[i];
+                u.len = plan.len[i];
                 u.split = unit - unit_prefix[i];
                 u.nsplit = unit_prefix[i + 1] - unit_prefix[i];
                 // the request's pages are shared out evenly among its units (no ragged last unit)
@@ -573,15 +688,19 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
                 u.t_end = min(u.len, u.t_begin + unit_pages * kPageSize);
                 u.ticket = i * p.Hkv + u.kvh;
                 u.slot = di;
-                const int beg = p.decode_page_indptr[i];
+                const int beg = plan.indptr[i];
                 u.pages = p.decode_pages + beg;
-                ok = (u.len + kPageSize - 1) / kPageSize <= p.decode_page_indptr[i + 1] - beg;
+                ok = (u.len + kPageSize - 1) / kPageSize <= plan.indptr[i + 1] - beg;
             }
             if (!ok) {
-                if (lane == 0) report(p.ctrl, SW_ERR_OUT_OF_RANGE, kSiteAttnLen, u.q_row);
-                continue;
+                if (lane == 0) {
+                    report(p.ctrl, SW_ERR_OUT_OF_RANGE, kSiteAttnLen, u.q_row);
+                    next_item = fixed_items + atomicAdd(&p.ctrl[kCtrWork], 1);
+                }
+            } else if (!run_unit<D>(&kvp_map, p, u, ring, fixed_items, next_item)) {
+                break;
             }
-            if (!run_unit<D>(&kv_map, p, u, ring)) break;
+            item = __shfl_sync(0xffffffffu, next_item, 0);
         }
     }
 
@@ -629,7 +748,7 @@ cudaError_t configure_kernels(int head_dim) {
                                 (int)mixed_attn_smem_bytes(128));
 }
 
-cudaError_t launch_mixed_attn(int head_dim, const CUtensorMap& kv_map, const CUtensorMap& q_map, const MixedParams& p,
+cudaError_t launch_mixed_attn(int head_dim, const KvMaps& kv_maps, const CUtensorMap& q_map, const MixedParams& p,
                               int num_sms, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)num_sms);
@@ -641,8 +760,8 @@ cudaError_t launch_mixed_attn(int head_dim, const CUtensorMap& kv_map, const CUt
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (head_dim == 64) return cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<64>, kv_map, q_map, p);
-    return cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<128>, kv_map, q_map, p);
+    if (head_dim == 64) return cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<64>, kv_maps.tile, kv_maps.page, q_map, p);
+    return cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<128>, kv_maps.tile, kv_maps.page, q_map, p);
 }
 
 }  // namespace sw

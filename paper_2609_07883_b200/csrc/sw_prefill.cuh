@@ -633,7 +633,8 @@ __device__ __forceinline__ void prefill_phase(const CUtensorMap* kv_map, const C
             } else if (warp == 2) {
                 if (it.j1 > it.j0) pf_sanitize<D>(p, sh, it, san_kv_it);
             } else {
-                if (lane == 0) next[iter & 1] = atomicAdd(&p.ctrl[kCtrPrefill], 1);
+                // entries 0 .. gridDim.x-1 are the CTAs' first ones; the counter hands out the rest
+                if (lane == 0) next[iter & 1] = (int)gridDim.x + atomicAdd(&p.ctrl[kCtrPrefill], 1);
             }
             if (!piece_sync()) break;
             entry = next[iter & 1];

@@ -33,9 +33,7 @@ static_assert(kScratchBytes <= SW_STATIC_SCRATCH_BYTES, "the header states the s
 // In host code this name is only a stand-in for the symbol; the device address comes from cudaGetSymbolAddress.
 static __device__ __align__(256) unsigned char g_static_scratch[SW_STATIC_SCRATCH_BYTES];
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+using sw::EncodeTiledFn;
 
 struct DeviceState {
     bool ready = false;
@@ -113,17 +111,9 @@ extern "C" sw_status sw_decode_attn_static(const sw_layout* layout, int device, 
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 
-    // tensor map of the pool, encoded on the stack for this call
-    CUtensorMap kv_map;
-    const cuuint64_t dims[4] = {(cuuint64_t)l.head_dim, (cuuint64_t)sw::kPageSize, (cuuint64_t)2 * l.num_kv_heads,
-                                (cuuint64_t)l.num_pages};
-    const cuuint64_t strides[3] = {(cuuint64_t)l.head_dim * 2, (cuuint64_t)sw::kPageSize * l.head_dim * 2,
-                                   (cuuint64_t)2 * l.num_kv_heads * sw::kPageSize * l.head_dim * 2};
-    const cuuint32_t box[4] = {64, (cuuint32_t)sw::kPageSize, 1, 1};
-    const cuuint32_t elem_strides[4] = {1, 1, 1, 1};
-    CUresult r = st->encode(&kv_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(kv_pool), dims, strides, box,
-                            elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    // tensor maps of the pool, encoded on the stack for this call
+    sw::KvMaps kv_maps;
+    CUresult r = sw::encode_kv_maps(st->encode, l, kv_pool, &kv_maps);
     if (r != CUDA_SUCCESS) return sw_fail(SW_ERR_CUDA, "cuTensorMapEncodeTiled(kv pool) failed with CUresult %d", (int)r);
 
     // the array keeps whatever the previous call left: counters and tickets must start at zero
@@ -151,6 +141,6 @@ extern "C" sw_status sw_decode_attn_static(const sw_layout* layout, int device, 
     p.part_o = reinterpret_cast<float*>(st->scratch + kOffPartO);
     p.max_items = kStaticMaxItems;
     p.target_items = kStaticTargetItems;
-    SW_CUDA(sw::launch_mixed_attn(l.head_dim, kv_map, kv_map, p, st->num_sms, s));
+    SW_CUDA(sw::launch_mixed_attn(l.head_dim, kv_maps, kv_maps.tile, p, st->num_sms, s));
     return SW_OK;
 }
