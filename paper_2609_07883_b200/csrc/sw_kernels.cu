@@ -117,11 +117,20 @@ struct Geo {
 };
 
 constexpr int kOneRoundMaxPages = 48;  // longest unit (pages) for which one round of units is planned
+constexpr int kPlanCounters = 8;       // shared counters of the plan's block sums, zeroed in the kernel prologue
+// When the CTAs of a single wave of prefill entries turn to decode units: a fixed start-up plus a time per 128-key
+// step of the longest entry (measured with the other CTAs streaming decode pages at the same time), and the rate at
+// which the decode units stream the pool meanwhile.
+#ifndef SW_LATE_STEP_US
+#define SW_LATE_STEP_US 2.2f
+#endif
+constexpr float kLateBaseUs = 1.0f, kLateStepUs = SW_LATE_STEP_US;
+constexpr float kDecodeBytesPerUs = 6.2e6f;
 struct Plan {
     const int* len;     // shared-memory copies of the context lengths and page-list offsets
     const int* indptr;
-    int split_tokens;   // tokens per split-KV unit (multiple of the page size)
-    int decode_units;   // sum over requests of ceil(len / split_tokens)
+    bool two_sizes;     // large units handed out by index to the early CTAs, small ones pulled by the late CTAs only
+    int decode_units;   // units of all requests
     int total_items;
 };
 
@@ -157,11 +166,39 @@ __device__ __forceinline__ int block_sum(int v, int* ctr) {
     return *reinterpret_cast<volatile int*>(ctr);
 }
 
+// One-class unit size: pages per unit when `warps_per_head` warps share `total_pages`.  Small batches are
+// latency-bound: one round of units, as many as there are warps, gets every warp streaming at once.  Large batches are
+// bandwidth-bound: a few rounds of smaller units shorten the tail.  Every request adds at most one ragged unit per
+// head, hence the "- n".
+__device__ __forceinline__ int plan_split_pages(const MixedParams& p, int total_pages, int warps_per_head) {
+    const int one_round = (total_pages + warps_per_head - 1) / warps_per_head;  // pages per unit if run in one round
+    const int rounds = one_round <= kOneRoundMaxPages ? 1 : (one_round <= 160 ? 2 : 4);
+    int units_target = max(1, rounds * warps_per_head - p.n);
+    units_target = min(units_target, max(1, p.target_items / p.Hkv));
+    return max((total_pages + units_target - 1) / units_target, kMinSplitTokens / kPageSize);
+}
+
+// CTAs that start with chunk-prefill work turn to decode units later than the others.
+struct LateJoin {
+    int ctas;   // how many CTAs (0 = none, gridDim.x = all: both plan like a decode-only launch)
+    float us;   // estimated delay of their first decode unit relative to the other CTAs' first
+};
+
 // Every CTA derives the same plan from the context lengths: no host planning, no extra launch.
-__device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix, int* len_s, int* indptr_s, int* scratch) {
+//
+// When some CTAs join late the plan may have two unit sizes (plan.two_sizes).  The decode phase is bandwidth-bound, so
+// by the time the late CTAs arrive the others have streamed about late.us * pages_per_us pages; what is left then is
+// shared evenly among all warps.  The first requests are cut into large units (streamed share + even share), one for
+// each warp of the early CTAs and handed out by index; the remaining requests are cut into small units (the even
+// share), which only the warps of the late CTAs pull from the counter.  Both counts are made to fit the warps that
+// run them, so that no warp starts a second unit.  If the early warps are nearly done by the time the late ones arrive,
+// the plan is sized for the early warps alone; with many requests per warp it falls back to units pulled by everybody.
+__device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix, int* len_s, int* indptr_s, int* scratch,
+                                          LateJoin late, float pages_per_us) {
     Plan plan;
     plan.len = len_s;
     plan.indptr = indptr_s;
+    plan.two_sizes = false;
     const int per_thread = (p.n + kThreads - 1) / kThreads;
     const int beg = min(p.n, (int)threadIdx.x * per_thread);
     const int end = min(p.n, beg + per_thread);
@@ -174,29 +211,75 @@ __device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix
         indptr_s[i] = p.decode_page_indptr[i];
     }
     if (threadIdx.x == 0 && p.n > 0) indptr_s[p.n] = p.decode_page_indptr[p.n];
-    const int total_pages = block_sum(pages_local, scratch + 64);  // counter zeroed in the kernel prologue
-    // Unit size.  Small batches are latency-bound: one round of units, as many as there are warps, gets every warp
-    // streaming at once.  Large batches are bandwidth-bound: a few rounds of smaller units shorten the tail.  Every
-    // request adds at most one ragged unit per head, hence the "- n".
-    const int per_head_warps = max(1, (int)gridDim.x * kWarps / p.Hkv);
-    const int one_round = (total_pages + per_head_warps - 1) / per_head_warps;  // pages per unit if run in one round
-    const int rounds = one_round <= kOneRoundMaxPages ? 1 : (one_round <= 160 ? 2 : 4);
-    int units_target = max(1, rounds * per_head_warps - p.n);
-    units_target = min(units_target, max(1, p.target_items / p.Hkv));
-    int split_pages = (total_pages + units_target - 1) / units_target;
-    split_pages = max(split_pages, kMinSplitTokens / kPageSize);
-    plan.split_tokens = split_pages * kPageSize;
+    int* ctr = scratch + 64;  // kPlanCounters counters zeroed in the kernel prologue, one per block sum
+    const int total_pages = block_sum(pages_local, ctr++);
+
+    const int G = (int)gridDim.x;
+    constexpr int kMinPages = kMinSplitTokens / kPageSize;
+    int split_a = 0, split_b = 0;  // pages per unit of the first requests / of the rest
+    int a_pages = 0x7fffffff;      // requests whose pages start below this (per head) are cut with split_a
+    if (late.ctas <= 0 || late.ctas >= G) {
+        split_a = split_b = plan_split_pages(p, total_pages, max(1, G * kWarps / p.Hkv));
+    } else {
+        const float early = (float)((G - late.ctas) * kWarps), all = (float)(G * kWarps);
+        const float pages = (float)total_pages * p.Hkv;
+        const float streamed = fminf(pages, pages_per_us * late.us);
+        const float even = (pages - streamed) / all;
+        // units and pages (per head) of the early warps and of the late ones; a request adds about half a ragged unit
+        const float a_units = early / p.Hkv, b_units = (all - early) / p.Hkv;
+        const float a_share = fminf((float)total_pages, a_units * (streamed / early + even));
+        const float b_share = (float)total_pages - a_share;
+        const float a_ragged = 0.6f * p.n * a_share / fmaxf(1.f, (float)total_pages);
+        const float b_ragged = 0.6f * p.n - a_ragged;
+        if (pages - streamed < (float)(late.ctas * kWarps * kMinPages)) {
+            split_a = split_b = plan_split_pages(p, total_pages, max(1, (G - late.ctas) * kWarps / p.Hkv));
+        } else if (a_ragged > 0.5f * a_units || b_ragged > 0.5f * b_units) {
+            split_a = split_b = plan_split_pages(p, total_pages, max(1, G * kWarps / p.Hkv));
+        } else {
+            split_a = max(kMinPages, (int)ceilf(a_share / (a_units - a_ragged)));
+            split_b = max(kMinPages, (int)ceilf(b_share / (b_units - b_ragged)));
+            a_pages = (int)a_share;
+            plan.two_sizes = true;
+        }
+    }
+    int pages_before = 0;
+    if (plan.two_sizes) {
+        int unused;
+        pages_before = block_exclusive_scan(pages_local, scratch + 16, &unused);
+        // count the units of either size and grow the size until they fit their warps (the estimates are rarely off)
+        const int a_units = (G - late.ctas) * kWarps / p.Hkv, b_units = late.ctas * kWarps / p.Hkv;
+        for (int pass = 0; pass < (kPlanCounters - 1) / 2; ++pass) {
+            int cnt_a = 0, cnt_b = 0, before = pages_before;
+            for (int i = beg; i < end; ++i) {
+                const int pg = len_s[i] > 0 ? (len_s[i] + kPageSize - 1) / kPageSize : 0;
+                if (before < a_pages) cnt_a += (pg + split_a - 1) / split_a; else cnt_b += (pg + split_b - 1) / split_b;
+                before += pg;
+            }
+            const int total_a = block_sum(cnt_a, ctr++);
+            const int total_b = block_sum(cnt_b, ctr++);
+            if (total_a <= a_units && total_b <= b_units) break;
+            if (total_a > a_units) split_a = (int)(((int64_t)split_a * total_a + a_units - 1) / a_units) + 1;
+            if (total_b > b_units) split_b = (int)(((int64_t)split_b * total_b + b_units - 1) / b_units) + 1;
+        }
+    }
     int units_local = 0;
     for (int i = beg; i < end; ++i) {
         const int len = len_s[i];
-        units_local += len > 0 ? (len + plan.split_tokens - 1) / plan.split_tokens : 0;
+        const int pg = len > 0 ? (len + kPageSize - 1) / kPageSize : 0;
+        const int split = pages_before < a_pages ? split_a : split_b;
+        units_local += (pg + split - 1) / split;
+        pages_before += pg;
     }
+    pages_before -= pages_local;
     int total_units = 0;
     int run = block_exclusive_scan(units_local, scratch, &total_units);
     for (int i = beg; i < end; ++i) {
         unit_prefix[i] = run;
         const int len = len_s[i];
-        run += len > 0 ? (len + plan.split_tokens - 1) / plan.split_tokens : 0;
+        const int pg = len > 0 ? (len + kPageSize - 1) / kPageSize : 0;
+        const int split = pages_before < a_pages ? split_a : split_b;
+        run += (pg + split - 1) / split;
+        pages_before += pg;
     }
     if (threadIdx.x == 0) unit_prefix[p.n] = total_units;
     __syncthreads();
@@ -360,7 +443,7 @@ __device__ __forceinline__ void merge_splits(const MixedParams& p, const Unit& u
 
 // Runs one unit; returns false if a bounded wait expired.
 template <int D>
-__device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const Unit& u, WarpRing<D>& ring, int fixed_items,
+__device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const Unit& u, WarpRing<D>& ring, int fixed_items, bool pulls,
                          int& next_item) {
     constexpr int KS = D / 16;  // k-slices of QK^T; also pairs of 8-wide output column tiles of PV
     const int lane = threadIdx.x & 31;
@@ -422,7 +505,7 @@ __device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const
     auto claim_next = [&]() {
         if (!claimed && issued >= npg) {
             claimed = true;
-            if (lane == 0) next_item = fixed_items + atomicAdd(&p.ctrl[kCtrWork], 1);
+            if (lane == 0) next_item = pulls ? fixed_items + atomicAdd(&p.ctrl[kCtrWork], 1) : 0x7fffffff;
         }
     };
     claim_next();
@@ -595,7 +678,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
 
     const bool tensor_prefill = p.C > 0;
     volatile int* misc = reinterpret_cast<volatile int*>(scratch + 32);  // [0] TMEM base, [1] abort flag, [2..3] ticket flags
-    if (threadIdx.x == 32) scratch[64] = 0;  // the plan's block-sum counter
+    if (threadIdx.x >= 32 && threadIdx.x < 32 + kPlanCounters) scratch[64 + threadIdx.x - 32] = 0;  // block-sum counters
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&kv_map);
         tma_prefetch_desc(&kvp_map);
@@ -618,9 +701,12 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     // The first prefill entry of a CTA is its own index and the first decode unit of a warp is fixed as well: neither
     // waits for a counter.  CTAs that start with prefill work take all their decode units from the counter.
     int prefill_ctas = 0;
+    LateJoin late{0, 0.f};
     if (tensor_prefill) {
         const PfPlan pplan = pf_make_plan(p);
         prefill_ctas = min(pplan.n_entries, (int)gridDim.x);
+        late.ctas = prefill_ctas;
+        late.us = kLateBaseUs + kLateStepUs * ((pf_steps_of_rank(p, pplan.n_tp, 0) + pplan.pieces - 1) / pplan.pieces);
         const int first_entry = blockIdx.x;
         if (first_entry < pplan.n_entries) {  // CTA-uniform: this CTA has prefill work
             if (warp == 1) {
@@ -649,7 +735,8 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     }
 
     const Plan plan = make_plan(p, unit_prefix, reinterpret_cast<int*>(smem + Geo<D>::kLenOffset),
-                                reinterpret_cast<int*>(smem + Geo<D>::kIndptrOffset), scratch);
+                                reinterpret_cast<int*>(smem + Geo<D>::kIndptrOffset), scratch, late,
+                                kDecodeBytesPerUs / Geo<D>::kStageBytes);
     if (plan.total_items > p.max_items) {
         if (threadIdx.x == 0) report(p.ctrl, SW_ERR_WORKSPACE, kSiteScratch, plan.total_items);
     } else {
@@ -658,6 +745,8 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
         ring.bar = base + Geo<D>::kBarOffset + warp * kStages * 8;
         ring.it = 0;
         const int fixed_items = ((int)gridDim.x - prefill_ctas) * kWarps;  // units handed out without the counter
+        // with two unit sizes the early CTAs run their one large unit each and leave the counter to the late CTAs
+        const bool pulls = !plan.two_sizes || (int)blockIdx.x < prefill_ctas;
         int item = ((int)blockIdx.x - prefill_ctas) * kWarps + warp;
         if ((int)blockIdx.x < prefill_ctas) {
             if (lane == 0) item = fixed_items + atomicAdd(&p.ctrl[kCtrWork], 1);
@@ -695,9 +784,9 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
             if (!ok) {
                 if (lane == 0) {
                     report(p.ctrl, SW_ERR_OUT_OF_RANGE, kSiteAttnLen, u.q_row);
-                    next_item = fixed_items + atomicAdd(&p.ctrl[kCtrWork], 1);
+                    next_item = pulls ? fixed_items + atomicAdd(&p.ctrl[kCtrWork], 1) : 0x7fffffff;
                 }
-            } else if (!run_unit<D>(&kvp_map, p, u, ring, fixed_items, next_item)) {
+            } else if (!run_unit<D>(&kvp_map, p, u, ring, fixed_items, pulls, next_item)) {
                 break;
             }
             item = __shfl_sync(0xffffffffu, next_item, 0);
