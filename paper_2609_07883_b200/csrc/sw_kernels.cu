@@ -126,6 +126,7 @@ constexpr int kPlanCounters = 8;       // shared counters of the plan's block su
 #endif
 constexpr float kLateBaseUs = 1.0f, kLateStepUs = SW_LATE_STEP_US;
 constexpr float kDecodeBytesPerUs = 6.2e6f;
+constexpr float kCtaBytesPerUs = 1.0e5f;  // what one CTA's ring of page copies sustains on its own
 struct Plan {
     const int* len;     // shared-memory copies of the context lengths and page-list offsets
     const int* indptr;
@@ -192,7 +193,8 @@ struct LateJoin {
 // each warp of the early CTAs and handed out by index; the remaining requests are cut into small units (the even
 // share), which only the warps of the late CTAs pull from the counter.  Both counts are made to fit the warps that
 // run them, so that no warp starts a second unit.  If the early warps are nearly done by the time the late ones arrive,
-// the plan is sized for the early warps alone; with many requests per warp it falls back to units pulled by everybody.
+// the plan is sized for the early warps alone; if their head start is small or there are many requests per warp, it
+// falls back to units of one size pulled by everybody.
 __device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix, int* len_s, int* indptr_s, int* scratch,
                                           LateJoin late, float pages_per_us) {
     Plan plan;
@@ -223,7 +225,9 @@ __device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix
     } else {
         const float early = (float)((G - late.ctas) * kWarps), all = (float)(G * kWarps);
         const float pages = (float)total_pages * p.Hkv;
-        const float streamed = fminf(pages, pages_per_us * late.us);
+        // few early CTAs cannot keep the memory system busy: their copies in flight bound the rate
+        const float rate = fminf(pages_per_us, pages_per_us * (float)(G - late.ctas) * (kCtaBytesPerUs / kDecodeBytesPerUs));
+        const float streamed = fminf(pages, rate * late.us);
         const float even = (pages - streamed) / all;
         // units and pages (per head) of the early warps and of the late ones; a request adds about half a ragged unit
         const float a_units = early / p.Hkv, b_units = (all - early) / p.Hkv;
@@ -233,7 +237,9 @@ __device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix
         const float b_ragged = 0.6f * p.n - a_ragged;
         if (pages - streamed < (float)(late.ctas * kWarps * kMinPages)) {
             split_a = split_b = plan_split_pages(p, total_pages, max(1, (G - late.ctas) * kWarps / p.Hkv));
-        } else if (a_ragged > 0.5f * a_units || b_ragged > 0.5f * b_units) {
+        } else if (streamed < 0.25f * pages || a_ragged > 0.25f * a_units || b_ragged > 0.25f * b_units) {
+            // The head start is small next to the whole phase, or there are too many requests per warp for one even
+            // unit each: units of one size pulled by every warp balance better.
             split_a = split_b = plan_split_pages(p, total_pages, max(1, G * kWarps / p.Hkv));
         } else {
             split_a = max(kMinPages, (int)ceilf(a_share / (a_units - a_ragged)));
