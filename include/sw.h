@@ -100,8 +100,18 @@ sw_status sw_kv_append(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const 
 sw_status sw_mixed_attn_run(sw_ctx* ctx, const void* kv_pool, const sw_batch* batch, const void* q, void* out,
                             float* lse, void* stream);
 
+/* KV manager step and executor step of one iteration in ONE kernel launch: what sw_kv_append followed by
+ * sw_mixed_attn_run computes, without the second launch and the gap between the two.  Every CTA of the persistent
+ * grid first writes its share of the k_new / v_new rows into the pool; the chunk-prefill tiles that reach into the
+ * chunk's own keys and the decode units that reach a request's last page wait (bounded) until every CTA has done so.
+ * Arguments as for the two calls.  Contract beyond theirs: no page of a decode request other than its last, and no
+ * page below the chunk's first row, is written by this call (true of any page table in which requests own their
+ * pages, shared prompt prefixes included).  Asynchronous. */
+sw_status sw_mixed_iteration_run(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const void* k_new, const void* v_new,
+                                 const void* q, void* out, float* lse, void* stream);
+
 /* The same iteration from HOST buffers: copies q / k_new / v_new and the page tables to the device (into the
- * workspace), runs sw_kv_append + sw_mixed_attn_run, copies `out` (and lse if non-NULL) back and waits.
+ * workspace), runs sw_mixed_iteration_run, copies `out` (and lse if non-NULL) back and waits.
  * All pointers inside `h_batch` and h_q / h_k_new / h_v_new / h_out / h_lse are HOST pointers (pinned memory
  * makes the copies asynchronous); kv_pool stays a device pointer. */
 sw_status sw_mixed_iteration_host(sw_ctx* ctx, void* kv_pool, const sw_batch* h_batch, const void* h_q,

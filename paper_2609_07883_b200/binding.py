@@ -47,7 +47,7 @@ class sw_choice(C.Structure):
                 ("queries", C.c_int32)]
 
 
-EXPORTS = ["sw_workspace_bytes", "sw_create", "sw_destroy", "sw_kv_append", "sw_mixed_attn_run",
+EXPORTS = ["sw_workspace_bytes", "sw_create", "sw_destroy", "sw_kv_append", "sw_mixed_attn_run", "sw_mixed_iteration_run",
            "sw_mixed_iteration_host", "sw_cost_probe", "sw_check_status", "sw_cost_table_create",
            "sw_cost_table_destroy", "sw_cost_table_lookup", "sw_choose_chunk", "sw_last_error",
            "sw_decode_attn_static", "sw_selftest_wait_timeout"]
@@ -60,6 +60,7 @@ _lib.sw_destroy.argtypes = [_vp]
 _lib.sw_destroy.restype = None
 _lib.sw_kv_append.argtypes = [_vp, _vp, C.POINTER(sw_batch), _vp, _vp, _vp]
 _lib.sw_mixed_attn_run.argtypes = [_vp, _vp, C.POINTER(sw_batch), _vp, _vp, _vp, _vp]
+_lib.sw_mixed_iteration_run.argtypes = [_vp, _vp, C.POINTER(sw_batch), _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sw_mixed_iteration_host.argtypes = [_vp, _vp, C.POINTER(sw_batch), _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sw_cost_probe.argtypes = [_vp, C.POINTER(_vp), _i32, C.POINTER(sw_batch), _vp, _vp, _i32, _i32,
                                C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), _vp]
@@ -182,6 +183,11 @@ def sw_kv_append(ctx: Context, kv_pool, batch: DeviceBatch, k_new, v_new, stream
 def sw_mixed_attn_run(ctx: Context, kv_pool, batch: DeviceBatch, q, out, lse=None, stream=None) -> None:
     _check(_lib.sw_mixed_attn_run(ctx.handle, _ptr(kv_pool), C.byref(batch.struct), _ptr(q), _ptr(out), _ptr(lse),
                                   _stream_handle(stream)), "sw_mixed_attn_run")
+
+
+def sw_mixed_iteration_run(ctx: Context, kv_pool, batch: DeviceBatch, k_new, v_new, q, out, lse=None, stream=None) -> None:
+    _check(_lib.sw_mixed_iteration_run(ctx.handle, _ptr(kv_pool), C.byref(batch.struct), _ptr(k_new), _ptr(v_new), _ptr(q),
+                                       _ptr(out), _ptr(lse), _stream_handle(stream)), "sw_mixed_iteration_run")
 
 
 def sw_mixed_iteration_host(ctx: Context, kv_pool, host_struct: sw_batch, h_q, h_k_new, h_v_new, h_out, h_lse=None,

@@ -220,14 +220,17 @@ sw_status sw_kv_append(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const 
     return SW_OK;
 }
 
-sw_status sw_mixed_attn_run(sw_ctx* ctx, const void* kv_pool, const sw_batch* batch, const void* q, void* out, float* lse,
-                            void* stream) {
-    sw_status st = check_batch(ctx, batch, "sw_mixed_attn_run");
+namespace {
+// The attention launch; with k_new / v_new non-null the same launch first writes those rows into the pool.
+sw_status run_mixed(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const void* k_new, const void* v_new, const void* q,
+                    void* out, float* lse, void* stream, const char* who) {
+    sw_status st = check_batch(ctx, batch, who);
     if (st != SW_OK) return st;
     if (batch->chunk_len + batch->num_decode == 0) return SW_OK;
-    if (!kv_pool || !q || !out) return sw_fail(SW_ERR_INVALID_ARG, "sw_mixed_attn_run: null tensor");
-    if (((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) & 15) != 0)
-        return sw_fail(SW_ERR_INVALID_ARG, "sw_mixed_attn_run: q and out must be 16-byte aligned");
+    if (!kv_pool || !q || !out) return sw_fail(SW_ERR_INVALID_ARG, "%s: null tensor", who);
+    if (((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(k_new) |
+          reinterpret_cast<uintptr_t>(v_new)) & 15) != 0)
+        return sw_fail(SW_ERR_INVALID_ARG, "%s: tensors must be 16-byte aligned", who);
     const sw::KvMaps* kv_maps = nullptr;
     st = kv_map_for(ctx, kv_pool, &kv_maps);
     if (st != SW_OK) return st;
@@ -250,6 +253,11 @@ sw_status sw_mixed_attn_run(sw_ctx* ctx, const void* kv_pool, const sw_batch* ba
     p.q = static_cast<const __nv_bfloat16*>(q);
     p.out = static_cast<__nv_bfloat16*>(out);
     p.lse = lse;
+    if (k_new) {
+        p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+        p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+        p.pool = static_cast<__nv_bfloat16*>(kv_pool);
+    }
     p.ctrl = reinterpret_cast<int32_t*>(ctx->ws + ctx->w.ctrl);
     p.tickets = reinterpret_cast<int32_t*>(ctx->ws + ctx->w.tickets);
     p.part_ml = reinterpret_cast<float*>(ctx->ws + ctx->w.part_ml);
@@ -274,6 +282,18 @@ sw_status sw_mixed_attn_run(sw_ctx* ctx, const void* kv_pool, const sw_batch* ba
     }
     SW_CUDA(sw::launch_mixed_attn(l.head_dim, *kv_maps, q_map, p, ctx->num_sms, static_cast<cudaStream_t>(stream)));
     return SW_OK;
+}
+}  // namespace
+
+sw_status sw_mixed_attn_run(sw_ctx* ctx, const void* kv_pool, const sw_batch* batch, const void* q, void* out, float* lse,
+                            void* stream) {
+    return run_mixed(ctx, const_cast<void*>(kv_pool), batch, nullptr, nullptr, q, out, lse, stream, "sw_mixed_attn_run");
+}
+
+sw_status sw_mixed_iteration_run(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const void* k_new, const void* v_new,
+                                 const void* q, void* out, float* lse, void* stream) {
+    if (!k_new || !v_new) return sw_fail(SW_ERR_INVALID_ARG, "sw_mixed_iteration_run: null tensor");
+    return run_mixed(ctx, kv_pool, batch, k_new, v_new, q, out, lse, stream, "sw_mixed_iteration_run");
 }
 
 sw_status sw_mixed_iteration_host(sw_ctx* ctx, void* kv_pool, const sw_batch* hb, const void* h_q, const void* h_k_new,
@@ -320,10 +340,9 @@ sw_status sw_mixed_iteration_host(sw_ctx* ctx, void* kv_pool, const sw_batch* hb
     db.decode_kv_len = d_len;
     db.decode_page_indptr = d_indptr;
     db.decode_pages = d_dec_pages;
-    st = sw_kv_append(ctx, kv_pool, &db, ws + ctx->w.st_k, ws + ctx->w.st_v, stream);
-    if (st != SW_OK) return st;
     float* d_lse = h_lse ? reinterpret_cast<float*>(ws + ctx->w.st_lse) : nullptr;
-    st = sw_mixed_attn_run(ctx, kv_pool, &db, ws + ctx->w.st_q, ws + ctx->w.st_out, d_lse, stream);
+    st = sw_mixed_iteration_run(ctx, kv_pool, &db, ws + ctx->w.st_k, ws + ctx->w.st_v, ws + ctx->w.st_q, ws + ctx->w.st_out,
+                                d_lse, stream);
     if (st != SW_OK) return st;
     SW_CUDA(cudaMemcpyAsync(h_out, ws + ctx->w.st_out, q_bytes, cudaMemcpyDeviceToHost, s));
     if (h_lse) SW_CUDA(cudaMemcpyAsync(h_lse, d_lse, (size_t)rows * l.num_q_heads * 4, cudaMemcpyDeviceToHost, s));

@@ -20,7 +20,8 @@ constexpr int kMaxCtas = 192;           // persistent CTAs (one per SM) the scra
 constexpr int kMaxChunk = 65536;        // chunk tokens per iteration (256-row groups are planned in shared memory)
 
 // Control words at the start of the workspace.
-enum CtrlWord { kCtrWork = 0, kCtrDone = 1, kCtrStatus = 2, kCtrDetail = 3, kCtrPrefill = 4, kCtrWords = 64 };
+// kCtrAppend counts the CTAs of a fused launch that have finished writing their share of the new K/V rows.
+enum CtrlWord { kCtrWork = 0, kCtrDone = 1, kCtrStatus = 2, kCtrDetail = 3, kCtrPrefill = 4, kCtrAppend = 5, kCtrWords = 64 };
 
 // Device-detected problem locators written to kCtrDetail (high byte = site, low 24 bits = index).
 enum DetailSite { kSiteAppendPage = 1, kSiteAppendLen = 2, kSiteAttnLen = 3, kSiteAttnPage = 4, kSiteWait = 5,
@@ -42,6 +43,11 @@ struct MixedParams {
     const __nv_bfloat16* q;
     __nv_bfloat16* out;
     float* lse;
+    // fused KV append (sw_mixed_iteration_run): the rows' new K/V and the pool to write them to; null when the append
+    // ran as a launch of its own
+    const __nv_bfloat16* k_new;
+    const __nv_bfloat16* v_new;
+    __nv_bfloat16* pool;
     // scratch
     int32_t* ctrl;
     int32_t* tickets;   // [max_decode * Hkv]

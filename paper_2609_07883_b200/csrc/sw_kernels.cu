@@ -25,15 +25,12 @@ __device__ __forceinline__ void report(int32_t* ctrl, int code, int site, int in
 // ---------------------------------------------------------------------------------------------------------------
 // KV append
 // ---------------------------------------------------------------------------------------------------------------
-// One thread per (row, 16-byte piece of the row's Hkv*D elements); it copies that piece of K and of V.
-__global__ void sw_kv_append_kernel(const AppendParams p) {
-    // launched with programmatic stream serialization: it may start while the previous kernel (the attention of
-    // the previous iteration, possibly still reading this pool) drains; nothing is touched before this wait
-    grid_launch_dependents();
-    grid_dependency_wait();
+// One thread per (row, 16-byte piece of the row's Hkv*D elements); it copies that piece of K and of V.  `first` and
+// `stride` spread the pieces over the calling threads.
+__device__ __forceinline__ void append_rows(const AppendParams& p, int64_t first, int64_t stride) {
     const int pieces_per_row = p.Hkv * p.D / 8;
     const int64_t total = (int64_t)(p.C + p.n) * pieces_per_row;
-    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+    for (int64_t idx = first; idx < total; idx += stride) {
         const int row = (int)(idx / pieces_per_row);
         const int piece = (int)(idx % pieces_per_row);
         int64_t pos;
@@ -77,6 +74,14 @@ __global__ void sw_kv_append_kernel(const AppendParams p) {
     }
 }
 
+__global__ void sw_kv_append_kernel(const AppendParams p) {
+    // launched with programmatic stream serialization: it may start while the previous kernel (the attention of
+    // the previous iteration, possibly still reading this pool) drains; nothing is touched before this wait
+    grid_launch_dependents();
+    grid_dependency_wait();
+    append_rows(p, (int64_t)blockIdx.x * blockDim.x + threadIdx.x, (int64_t)gridDim.x * blockDim.x);
+}
+
 cudaError_t launch_kv_append(const AppendParams& p, cudaStream_t stream) {
     const int64_t total = (int64_t)(p.C + p.n) * (p.Hkv * p.D / 8);
     if (total == 0) return cudaSuccess;
@@ -94,6 +99,29 @@ cudaError_t launch_kv_append(const AppendParams& p, cudaStream_t stream) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, sw_kv_append_kernel, p);
+}
+
+// Fused launches (append and attention in one kernel): every CTA writes its share of the new K/V rows at the start of
+// the kernel and then adds one to a counter.  A page that can hold one of those rows (the last page of a decode
+// request; the chunk's own keys) is not fetched before the counter shows every CTA's share.  The grid is one CTA per
+// SM, so all CTAs are resident and the wait is short; it is bounded all the same.  Whole-warp call; false when the
+// wait ran out.
+__device__ __forceinline__ bool wait_append(const MixedParams& p) {
+    if (p.pool == nullptr) return true;
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) {
+        const long long t0 = clock64();
+        while (ld_acquire_gpu(&p.ctrl[kCtrAppend]) < (int)gridDim.x) {
+            if (clock64() - t0 > kWaitBudgetCycles) {
+                ok = 0;
+                break;
+            }
+            __nanosleep(64);
+        }
+    }
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    fence_proxy_async_global();  // the rows were written with plain stores and are read through TMA
+    return ok != 0;
 }
 
 // ---------------------------------------------------------------------------------------------------------------
@@ -126,7 +154,7 @@ constexpr int kPlanCounters = 8;       // shared counters of the plan's block su
 #endif
 constexpr float kLateBaseUs = 1.0f, kLateStepUs = SW_LATE_STEP_US;
 constexpr float kDecodeBytesPerUs = 6.2e6f;
-constexpr float kCtaBytesPerUs = 1.0e5f;  // what one CTA's ring of page copies sustains on its own
+constexpr int kMinEarlyCtas = 64;  // CTAs whose rings of page copies keep the memory system busy on their own
 struct Plan {
     const int* len;     // shared-memory copies of the context lengths and page-list offsets
     const int* indptr;
@@ -193,8 +221,8 @@ struct LateJoin {
 // each warp of the early CTAs and handed out by index; the remaining requests are cut into small units (the even
 // share), which only the warps of the late CTAs pull from the counter.  Both counts are made to fit the warps that
 // run them, so that no warp starts a second unit.  If the early warps are nearly done by the time the late ones arrive,
-// the plan is sized for the early warps alone; if their head start is small or there are many requests per warp, it
-// falls back to units of one size pulled by everybody.
+// the plan is sized for the early warps alone; if the early CTAs are few, their head start is small or there are many
+// requests per warp, it falls back to units of one size pulled by everybody.
 __device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix, int* len_s, int* indptr_s, int* scratch,
                                           LateJoin late, float pages_per_us) {
     Plan plan;
@@ -225,9 +253,7 @@ __device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix
     } else {
         const float early = (float)((G - late.ctas) * kWarps), all = (float)(G * kWarps);
         const float pages = (float)total_pages * p.Hkv;
-        // few early CTAs cannot keep the memory system busy: their copies in flight bound the rate
-        const float rate = fminf(pages_per_us, pages_per_us * (float)(G - late.ctas) * (kCtaBytesPerUs / kDecodeBytesPerUs));
-        const float streamed = fminf(pages, rate * late.us);
+        const float streamed = fminf(pages, pages_per_us * late.us);
         const float even = (pages - streamed) / all;
         // units and pages (per head) of the early warps and of the late ones; a request adds about half a ragged unit
         const float a_units = early / p.Hkv, b_units = (all - early) / p.Hkv;
@@ -235,11 +261,14 @@ __device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix
         const float b_share = (float)total_pages - a_share;
         const float a_ragged = 0.6f * p.n * a_share / fmaxf(1.f, (float)total_pages);
         const float b_ragged = 0.6f * p.n - a_ragged;
-        if (pages - streamed < (float)(late.ctas * kWarps * kMinPages)) {
+        if (G - late.ctas < kMinEarlyCtas || streamed < 0.25f * pages) {
+            // Too few early CTAs to keep the memory system busy on their own (the estimate of what they stream would
+            // not hold), or a head start that is small next to the whole phase: one unit size, every warp pulls.
+            split_a = split_b = plan_split_pages(p, total_pages, max(1, G * kWarps / p.Hkv));
+        } else if (pages - streamed < (float)(late.ctas * kWarps * kMinPages)) {
             split_a = split_b = plan_split_pages(p, total_pages, max(1, (G - late.ctas) * kWarps / p.Hkv));
-        } else if (streamed < 0.25f * pages || a_ragged > 0.25f * a_units || b_ragged > 0.25f * b_units) {
-            // The head start is small next to the whole phase, or there are too many requests per warp for one even
-            // unit each: units of one size pulled by every warp balance better.
+        } else if (a_ragged > 0.25f * a_units || b_ragged > 0.25f * b_units) {
+            // too many requests per warp for one even unit each: units pulled by every warp balance better
             split_a = split_b = plan_split_pages(p, total_pages, max(1, G * kWarps / p.Hkv));
         } else {
             split_a = max(kMinPages, (int)ceilf(a_share / (a_units - a_ragged)));
@@ -491,6 +520,7 @@ __device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const
 
     int ids = 0;
     int issued = 0;
+    bool append_timeout = false;
     const uint32_t it0 = ring.it;  // ring position of this unit's first page
     auto issue_next = [&]() {
         if ((issued & 31) == 0) {
@@ -500,6 +530,11 @@ __device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const
         const int page = __shfl_sync(0xffffffffu, ids, issued & 31);
         if (page < 0 || (int64_t)page >= p.num_pages) {
             if (lane == 0) report(p.ctrl, SW_ERR_OUT_OF_RANGE, kSiteAttnPage, u.q_row);
+        }
+        // the request's last page holds the row this iteration appends
+        if (p.pool != nullptr && (pg0 + issued + 1) * kPageSize >= u.len && !wait_append(p)) {
+            if (lane == 0) report(p.ctrl, SW_ERR_DEVICE_TIMEOUT, kSiteWait, u.q_row);
+            append_timeout = true;
         }
         issue_page<D>(kvp_map, ring, it0 + issued, page, u.kvh);
         ++issued;
@@ -517,6 +552,7 @@ __device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const
     claim_next();
 
     for (int k = 0; k < npg; ++k) {
+        if (append_timeout) return false;
         const uint32_t stage = ring.it % kStages;
         const uint32_t parity = (ring.it / kStages) & 1;
         const uint32_t sK = ring.buf + stage * Geo<D>::kStageBytes;
@@ -701,6 +737,30 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     // kernels of the stream wrote (the pool after the KV append, q, the page tables): wait for them to finish.
     grid_dependency_wait();
     grid_launch_dependents();
+    if (p.pool != nullptr) {
+        // fused launch: this CTA's share of the new K/V rows, then its mark on the counter the readers wait for
+        AppendParams a;
+        a.Hkv = p.Hkv;
+        a.D = D;
+        a.num_pages = p.num_pages;
+        a.P = p.P;
+        a.C = p.C;
+        a.n = p.n;
+        a.prefill_pages = p.prefill_pages;
+        a.num_prefill_pages = p.num_prefill_pages;
+        a.decode_kv_len = p.decode_kv_len;
+        a.decode_page_indptr = p.decode_page_indptr;
+        a.decode_pages = p.decode_pages;
+        a.k_new = p.k_new;
+        a.v_new = p.v_new;
+        a.pool = p.pool;
+        a.ctrl = p.ctrl;
+        append_rows(a, (int64_t)blockIdx.x * kThreads + threadIdx.x, (int64_t)gridDim.x * kThreads);
+        fence_proxy_async_global();
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) atomicAdd(&p.ctrl[kCtrAppend], 1);
+    }
     __syncthreads();
 
     // chunk-prefill tiles first (long, tensor-bound); the decode units below fill the tail
@@ -807,6 +867,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
         if (done == (int)gridDim.x - 1) {
             p.ctrl[kCtrWork] = 0;
             p.ctrl[kCtrPrefill] = 0;
+            p.ctrl[kCtrAppend] = 0;
             p.ctrl[kCtrDone] = 0;
             __threadfence();
         }

@@ -183,6 +183,14 @@ __device__ __forceinline__ bool pf_produce(const CUtensorMap* kv_map, const CUte
                     tma_load_3d(sh.smem + G::kQOffset + t * G::kTileBytes + h * G::kHalfBytes, q_map, sh.bars + kBarQFull * 8,
                                 h * 64, it.kvh * p.group, it.tok0[t]);
     }
+    // fused launch: tiles that reach into the chunk's own keys wait until every CTA has written its share of them
+    if (p.pool != nullptr && it.j1 * 128 > p.P && !wait_append(p)) {
+        if (lane == 0) {
+            *sh.abort_flag = 1;
+            report(p.ctrl, SW_ERR_DEVICE_TIMEOUT, kSiteWait, it.item);
+        }
+        return false;
+    }
     const int npages = (p.P + p.C + kPageSize - 1) / kPageSize;
     auto page_of = [&](int j) { return (lane < 8 && j * 8 + lane < npages) ? p.prefill_pages[j * 8 + lane] : 0; };
     int id_next = page_of(it.j0);

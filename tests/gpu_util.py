@@ -50,6 +50,10 @@ class Runner:
     def attend(self):
         self.B.sw_mixed_attn_run(self.ctx, self.pool, self.dbatch, self.q, self.out, self.lse)
 
+    def iterate(self):
+        """Append and attention in one launch."""
+        self.B.sw_mixed_iteration_run(self.ctx, self.pool, self.dbatch, self.k_new, self.v_new, self.q, self.out, self.lse)
+
     def status(self):
         return self.B.sw_check_status(self.ctx, raise_on_error=False)
 

@@ -21,10 +21,13 @@ def gpu():
     return gpu_util
 
 
-def run_and_compare(gpu, oracle, batch, tensors, pairs=None, what=""):
+def run_and_compare(gpu, oracle, batch, tensors, pairs=None, what="", fused=False):
     r = gpu.Runner(batch, tensors)
-    r.append()
-    r.attend()
+    if fused:
+        r.iterate()
+    else:
+        r.append()
+        r.attend()
     out, lse = r.results()
     assert r.status() == (0, 0), f"{what}: device status {r.status()}"
     # oracle on its own copy of the pool, appended by the oracle
@@ -59,6 +62,55 @@ def test_ragged_small_cases(gpu, oracle, shape):
     batch = W.make_batch(shape, 160, lens, 37, 91, rng)
     t = W.host_tensors(batch, rng)
     run_and_compare(gpu, oracle, batch, t, what=f"ragged {shape}")
+
+
+@pytest.mark.parametrize("case", ["tiny", "ragged", "ragged_d64", "decode_only", "prefill_only", "long_split", "chat"])
+def test_fused_iteration_matches_oracle(gpu, oracle, case):
+    """Append and attention in one launch: the rows written at the start of the kernel are the ones the diagonal tiles
+    and every request's last page must see."""
+    rng = np.random.default_rng(77)
+    pairs = None
+    if case == "tiny":
+        batch = W.tiny_batch(rng)
+    elif case == "ragged":
+        batch = W.make_batch(W.AttnShape(8, 2, 128), 200, [1, 15, 16, 17, 31, 255, 256, 257, 700], 37, 91, rng)
+    elif case == "ragged_d64":
+        batch = W.make_batch(W.AttnShape(4, 4, 64), 200, [1, 16, 17, 333, 700], 128, 300, rng)
+    elif case == "decode_only":
+        batch = W.make_batch(W.TINY, 120, [5, 64, 300, 301, 1], 0, 0, rng)
+    elif case == "prefill_only":
+        batch = W.make_batch(W.TINY, 120, [], 200, 333, rng)
+    elif case == "long_split":
+        batch = W.make_batch(W.AttnShape(8, 2, 128), 1400, [20000, 3], 0, 0, rng)
+    else:
+        batch = W.chat_batch(n=64, chunk_len=512, prefix_len=512, rng=rng)
+        rows = rng.choice(batch.num_rows, size=96, replace=False)
+        pairs = [(int(r), int(rng.integers(batch.shape.num_q_heads))) for r in rows]
+        pairs += [(batch.chunk_len - 1, 0), (batch.chunk_len, 1), (batch.num_rows - 1, 2)]
+    t = W.host_tensors(batch, rng)
+    run_and_compare(gpu, oracle, batch, t, pairs=pairs, what=f"fused {case}", fused=True)
+
+
+def test_fused_iteration_repeated_with_new_rows(gpu, oracle):
+    """Several fused launches in a row on one context, each appending different rows at the same positions: a launch
+    that read a page before its rows were written would return the previous launch's values."""
+    rng = np.random.default_rng(78)
+    batch = W.make_batch(W.AttnShape(8, 2, 128), 400, [17, 256, 1000, 4000, 16], 64, 200, rng)
+    t = W.host_tensors(batch, rng)
+    r = gpu.Runner(batch, t)
+    for it in range(4):
+        t["k_new"] = W.normal_bf16_bits(rng, *t["k_new"].shape)
+        t["v_new"] = W.normal_bf16_bits(rng, *t["v_new"].shape)
+        r.k_new = gpu.bits_to_torch(t["k_new"], r.dev)
+        r.v_new = gpu.bits_to_torch(t["v_new"], r.dev)
+        r.iterate()
+        out, lse = r.results()
+        assert r.status() == (0, 0)
+        pool = t["pool"]
+        assert oracle.kv_append(pool, batch, t["k_new"], t["v_new"]) == 0
+        assert np.array_equal(gpu.torch_to_bits(r.pool), pool), f"launch {it}: pool differs after append"
+        ref, ref_lse, _ = oracle.mixed_attention(pool, batch, t["q"])
+        gpu.compare(out.reshape(-1, batch.shape.head_dim), lse.reshape(-1), ref, ref_lse, f"fused launch {it}")
 
 
 def test_decode_only_and_prefill_only(gpu, oracle):
