@@ -2,8 +2,8 @@
 
 Each iteration decodes one token for every active request and optionally processes one prefill chunk of the oldest
 pending request (Sec. 4.1); requests that arrive during an iteration become eligible at its end.  The chunk is chosen
-by ``sw_choose_chunk`` (Algorithm 1) from the measured cost table; the iteration itself is KV append + the mixed
-attention launch over a stack of ``layers`` KV pools, and the virtual clock advances by its measured device time.
+by ``sw_choose_chunk`` (Algorithm 1) from the measured cost table; the iteration itself is one launch per layer (KV append
+and mixed attention together) over a stack of ``layers`` KV pools, and the virtual clock advances by its measured device time.
 Orchestration and bookkeeping only: chunk choice, append and attention all run in the library.
 """
 from __future__ import annotations
@@ -56,7 +56,7 @@ class Request:
 
 def gpu_executor(ctx, pools, shape: W.AttnShape, c_max: int, max_decode: int, seed: int = W.SEED_BASE + 44):
     """Returns execute(batch) -> measured device nanoseconds of one iteration over the layer stack: per layer one
-    KV append and one mixed attention launch, timed with CUDA events on the current stream."""
+    launch that appends the new K/V rows and runs the mixed attention, timed with CUDA events on the current stream."""
     import torch
 
     from . import binding as B
@@ -76,8 +76,7 @@ def gpu_executor(ctx, pools, shape: W.AttnShape, c_max: int, max_decode: int, se
         rows = batch.num_rows
         ev0.record()
         for pool_t in pools:
-            B.sw_kv_append(ctx, pool_t, db, k_new[:rows], v_new[:rows])
-            B.sw_mixed_attn_run(ctx, pool_t, db, q[:rows], out[:rows])
+            B.sw_mixed_iteration_run(ctx, pool_t, db, k_new[:rows], v_new[:rows], q[:rows], out[:rows])
         ev1.record()
         ev1.synchronize()
         return int(ev0.elapsed_time(ev1) * 1e6)
@@ -87,10 +86,13 @@ def gpu_executor(ctx, pools, shape: W.AttnShape, c_max: int, max_decode: int, se
 
 def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, num_pages: int, policy: str = "sloweave",
               c_max: int = 4096, margin_ppm: int = 50_000, margin_abs_ns: int = 0, quantum: int = 16, max_decode: int = 512,
-              ctx_cap: int | None = None, seed: int = W.SEED_BASE + 44, log=None) -> dict:
+              ctx_cap: int | None = None, seed: int = W.SEED_BASE + 44, log=None, page_tables: bool = True,
+              ttft_slo_ms: float | None = None) -> dict:
     """Run the whole trace; returns statistics.  ``policy`` is "sloweave" or "fixed:<chunk>".  ``execute(batch)`` runs
     one iteration and returns its duration in ns (``gpu_executor`` for the CUDA path).  ``ctx_cap`` clamps the total
-    context passed to the table lookup to the table's last grid point."""
+    context passed to the table lookup to the table's last grid point.  ``page_tables=False`` hands ``execute`` a batch
+    without page lists (enough for a cost model that looks only at sizes; the simulator study runs that way).  With
+    ``ttft_slo_ms`` the result also counts the requests that meet both SLOs and the goodput (Sec. 4.3)."""
     from . import binding as B
 
     S = shape.page_size
@@ -138,8 +140,17 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
             c = min(fixed_chunk, remaining)
         else:
             q_eff = quantum if remaining >= quantum else 1   # the last few tokens of a prompt are below the quantum
-            ch = B.sw_choose_chunk(table if n else None, now, deadlines, total_ctx, head.prefilled if head else 0, remaining,
+            prefilled = head.prefilled if head else 0
+            ch = B.sw_choose_chunk(table if n else None, now, deadlines, total_ctx, prefilled, remaining,
                                    c_max=c_max, chunk_quantum=q_eff, margin_abs_ns=margin_abs_ns, margin_ppm=margin_ppm)
+            L = min(c_max, remaining)
+            if q_eff > 1 and L % q_eff and ch.chunk == L - L % q_eff:
+                # The quantum stopped just short of L.  If L itself fits the budget, take it: a prompt's last few tokens
+                # would otherwise cost a whole extra iteration.
+                fine = B.sw_choose_chunk(table if n else None, now, deadlines, total_ctx, prefilled, remaining, c_max=c_max,
+                                         chunk_quantum=1, margin_abs_ns=margin_abs_ns, margin_ppm=margin_ppm)
+                if fine.chunk == L:
+                    ch = fine
             c, flags, predicted = ch.chunk, ch.flags, ch.predicted_ns
         if n == 0 and c == 0:
             # nothing to run (memory stall with an idle GPU): wait for the next arrival or fail loudly
@@ -153,9 +164,12 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
         per = [(-(-int(L) // S)) for L in lens]
         indptr = np.zeros(n + 1, dtype=np.int32)
         indptr[1:] = np.cumsum(per)
-        dpages = np.concatenate([np.asarray(r.pages[:k], dtype=np.int32) for r, k in zip(active, per)]) if n else \
-            np.zeros(0, np.int32)
-        ppages = np.asarray(head.pages[: -(-(P + c) // S)], dtype=np.int32) if c > 0 else np.zeros(0, np.int32)
+        if page_tables:
+            dpages = np.concatenate([np.asarray(r.pages[:k], dtype=np.int32) for r, k in zip(active, per)]) if n else \
+                np.zeros(0, np.int32)
+            ppages = np.asarray(head.pages[: -(-(P + c) // S)], dtype=np.int32) if c > 0 else np.zeros(0, np.int32)
+        else:
+            dpages = ppages = np.zeros(0, np.int32)
         batch = W.MixedBatch(shape, num_pages, P, c, ppages, lens, indptr, dpages)
         dt = int(execute(batch))
         now += dt
@@ -207,7 +221,13 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
     ttft = np.array([r.first_token - r.arrival for r in reqs], dtype=np.float64) / MS
     p99_gap = np.array([np.percentile(r.gaps, 99) if r.gaps else 0.0 for r in reqs]) / MS
     duration_s = now / 1e9
+    slo = {}
+    if ttft_slo_ms is not None:
+        both = int(np.sum((ttft <= ttft_slo_ms) & (p99_gap <= tpot_ms)))
+        slo = {"ttft_slo_ms": ttft_slo_ms, "requests_meeting_both_slos": both, "slo_attainment": both / len(reqs),
+               "goodput_rps": both / duration_s, "throughput_rps": len(reqs) / duration_s}
     return {
+        **slo,
         "policy": policy, "tpot_ms": tpot_ms, "requests": len(reqs), "iterations": iters, "chunk_iterations": chunk_iters,
         "deadline_misses_with_chunk": misses_chunk, "deadline_misses_decode_only": misses_decode_only,
         "decode_infeasible_flags": infeasible_flags, "memory_stalls": stalled_for_memory,
