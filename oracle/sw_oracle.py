@@ -183,3 +183,60 @@ def analytic_table(n_values, c_max: int) -> Table:
         for e, c in enumerate(chunk_grid):
             cost[a, 0, 0, e] = analytic_cost_ns(n, int(c))
     return Table(n_values, [1 << 40], [1 << 30], chunk_grid, cost)
+
+
+# --------------------------------------------------------------------------------------------
+# telemetry residuals (Sec. 3.3 "Prediction error"; Sec. 5.1; Table 1 "Telemetry") — plain Python
+# --------------------------------------------------------------------------------------------
+class ResidualTable:
+    """Empirical high-percentile residual table: the margin delta(n, c) of Sec. 3.3 and the fallback signal of
+    Sec. 5.1, written out as their definitions.
+
+    * residual of an iteration = max(0, observed - predicted) (one-sided: only under-prediction costs a deadline);
+    * iterations are bucketed by (n, c): a value falls into the first bucket whose upper edge is >= it, values
+      beyond the last edge into the last bucket; a bucket keeps its most recent ``window`` residuals;
+    * percentile = nearest rank: the ceil(p * N)-th smallest of the N kept residuals (at least the first);
+    * a bucket with fewer than ``min_samples`` residuals contributes ``floor_ns``;
+    * delta(n, c) = the largest bucket percentile over all buckets (i, j) with i <= bucket(n) and j <= bucket(c), so
+      that the margin is nondecreasing in n and in c (the feasibility test must stay monotone, Proposition 1);
+    * the fallback signal is delta(n, c) > the configured margin.
+    """
+
+    def __init__(self, n_edges, c_edges, window: int):
+        self.n_edges = [int(x) for x in n_edges]
+        self.c_edges = [int(x) for x in c_edges]
+        self.window = int(window)
+        self.kept = [[[] for _ in self.c_edges] for _ in self.n_edges]
+        self.records = 0
+
+    @staticmethod
+    def bucket(value: int, edges) -> int:
+        for i, e in enumerate(edges):
+            if value <= e:
+                return i
+        return len(edges) - 1
+
+    def record(self, n: int, c: int, predicted_ns: int, observed_ns: int) -> None:
+        cell = self.kept[self.bucket(n, self.n_edges)][self.bucket(c, self.c_edges)]
+        cell.append(max(0, int(observed_ns) - int(predicted_ns)))
+        if len(cell) > self.window:
+            del cell[0]
+        self.records += 1
+
+    @staticmethod
+    def nearest_rank(values, percentile_ppm: int) -> int:
+        ordered = sorted(values)
+        rank = -(-percentile_ppm * len(ordered) // 1_000_000)   # ceil(p * N) in integers
+        return ordered[max(rank, 1) - 1]
+
+    def margin(self, n: int, c: int, percentile_ppm: int = 990_000, min_samples: int = 1, floor_ns: int = 0) -> int:
+        best = None
+        for i in range(self.bucket(n, self.n_edges) + 1):
+            for j in range(self.bucket(c, self.c_edges) + 1):
+                cell = self.kept[i][j]
+                v = self.nearest_rank(cell, percentile_ppm) if len(cell) >= max(min_samples, 1) else int(floor_ns)
+                best = v if best is None else max(best, v)
+        return best
+
+    def exceeds(self, n: int, c: int, configured_margin_ns: int, percentile_ppm: int = 990_000, min_samples: int = 1) -> bool:
+        return self.margin(n, c, percentile_ppm, min_samples, 0) > configured_margin_ns
