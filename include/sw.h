@@ -197,6 +197,39 @@ typedef struct {
     int32_t queries;      /* cost-model queries made by the bisection */
 } sw_choice;
 
+/* ---- telemetry (host only; no CUDA) --------------------------------------------------------------- */
+
+/* Residual table of the online feedback loop (Table 1 "Telemetry"; Sec. 3.3 "Prediction error"; Sec. 5.1).  Every
+ * iteration's predicted and observed duration is recorded; the one-sided residual max(0, observed - predicted) goes
+ * into the bucket of its (decode count n, chunk c).  n_edges / c_edges are strictly increasing UPPER edges: a value
+ * falls into the first bucket whose edge is >= it, values beyond the last edge into the last bucket.  A bucket keeps
+ * its most recent `window` residuals. */
+typedef struct sw_telemetry sw_telemetry;
+typedef struct {
+    int64_t records;         /* iterations recorded */
+    int64_t fallbacks;       /* of those, iterations the caller marked as decode-only fallbacks */
+    int64_t deadline_misses; /* of those, iterations recorded with a negative deadline slack */
+    int64_t max_residual_ns; /* largest residual seen */
+} sw_telemetry_totals;
+sw_status sw_telemetry_create(const int32_t* n_edges, int32_t num_n, const int32_t* c_edges, int32_t num_c, int32_t window,
+                              sw_telemetry** out);
+void sw_telemetry_destroy(sw_telemetry* t);
+/* slack_ns = earliest deadline - end of the iteration (negative = a missed deadline); fallback != 0 marks an
+ * iteration that ran decode-only because sw_telemetry_exceeds said so. */
+sw_status sw_telemetry_record(sw_telemetry* t, int32_t n, int32_t c, int64_t predicted_ns, int64_t observed_ns,
+                              int64_t slack_ns, int32_t fallback);
+/* The margin delta(n, c) to reserve (Sec. 3.3): the nearest-rank percentile (percentile_ppm of 1e6, e.g. 990000) of a
+ * bucket's residuals, floor_ns for a bucket with fewer than min_samples of them, maximised over all buckets at or
+ * below the bucket of (n, c) in both coordinates so that the margin is nondecreasing in n and in c (the feasibility
+ * test of Algorithm 1 has to stay monotone).  Pass the result as sw_chooser_params.margin_abs_ns. */
+sw_status sw_telemetry_margin(const sw_telemetry* t, int32_t n, int32_t c, int32_t percentile_ppm, int32_t min_samples,
+                              int64_t floor_ns, int64_t* margin_ns);
+/* Fallback signal (Sec. 5.1): *exceeds = 1 when that margin (with floor 0) is larger than configured_margin_ns; the
+ * scheduler then runs the iteration decode-only. */
+sw_status sw_telemetry_exceeds(const sw_telemetry* t, int32_t n, int32_t c, int32_t percentile_ppm, int32_t min_samples,
+                               int64_t configured_margin_ns, int32_t* exceeds);
+sw_status sw_telemetry_get_totals(const sw_telemetry* t, sw_telemetry_totals* out);
+
 /* Algorithm 1: P empty -> 0; L = min(C_max, remaining); A empty -> L; B = min_i(d_i) - now; upper-mid
  * bisection over [0, L] on T^ + delta <= B.  deadlines_ns are absolute next-token deadlines d_i = l_i + D_i
  * (HOST array, n_active entries).  remaining_prefill = 0 means no pending prefill. */

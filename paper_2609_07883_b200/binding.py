@@ -47,10 +47,16 @@ class sw_choice(C.Structure):
                 ("queries", C.c_int32)]
 
 
+class sw_telemetry_totals(C.Structure):
+    _fields_ = [("records", C.c_int64), ("fallbacks", C.c_int64), ("deadline_misses", C.c_int64),
+                ("max_residual_ns", C.c_int64)]
+
+
 EXPORTS = ["sw_workspace_bytes", "sw_create", "sw_destroy", "sw_kv_append", "sw_mixed_attn_run", "sw_mixed_iteration_run",
            "sw_mixed_iteration_host", "sw_cost_probe", "sw_check_status", "sw_cost_table_create",
            "sw_cost_table_destroy", "sw_cost_table_lookup", "sw_choose_chunk", "sw_last_error",
-           "sw_decode_attn_static", "sw_selftest_wait_timeout"]
+           "sw_decode_attn_static", "sw_selftest_wait_timeout", "sw_telemetry_create", "sw_telemetry_destroy",
+           "sw_telemetry_record", "sw_telemetry_margin", "sw_telemetry_exceeds", "sw_telemetry_get_totals"]
 
 _vp, _i32, _i64 = C.c_void_p, C.c_int32, C.c_int64
 _lib.sw_workspace_bytes.restype = C.c_size_t
@@ -70,6 +76,13 @@ _lib.sw_check_status.argtypes = [_vp, _vp, C.POINTER(_i32), C.POINTER(_i32)]
 _lib.sw_cost_table_create.argtypes = [C.POINTER(_i32), _i32, C.POINTER(_i64), _i32, C.POINTER(_i32), _i32,
                                       C.POINTER(_i32), _i32, C.POINTER(_i64), C.c_int, C.c_int, C.POINTER(_vp)]
 _lib.sw_cost_table_destroy.argtypes = [_vp]
+_lib.sw_telemetry_create.argtypes = [C.POINTER(_i32), _i32, C.POINTER(_i32), _i32, _i32, C.POINTER(_vp)]
+_lib.sw_telemetry_destroy.argtypes = [_vp]
+_lib.sw_telemetry_destroy.restype = None
+_lib.sw_telemetry_record.argtypes = [_vp, _i32, _i32, _i64, _i64, _i64, _i32]
+_lib.sw_telemetry_margin.argtypes = [_vp, _i32, _i32, _i32, _i32, _i64, C.POINTER(_i64)]
+_lib.sw_telemetry_exceeds.argtypes = [_vp, _i32, _i32, _i32, _i32, _i64, C.POINTER(_i32)]
+_lib.sw_telemetry_get_totals.argtypes = [_vp, C.POINTER(sw_telemetry_totals)]
 _lib.sw_cost_table_destroy.restype = None
 _lib.sw_cost_table_lookup.argtypes = [_vp, _i64, _i64, _i64, _i64, C.POINTER(_i64)]
 _lib.sw_choose_chunk.argtypes = [_vp, C.POINTER(sw_chooser_params), _i64, C.POINTER(_i64), _i32, _i64, _i32, _i32,
@@ -263,6 +276,47 @@ class CostTable:
     def close(self):
         if getattr(self, "handle", None) and _lib is not None:
             _lib.sw_cost_table_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        self.close()
+
+
+class Telemetry:
+    """Residual table of the online feedback loop (``sw_telemetry_*``)."""
+
+    def __init__(self, n_edges, c_edges, window: int = 256):
+        ne = np.ascontiguousarray(n_edges, dtype=np.int32)
+        ce = np.ascontiguousarray(c_edges, dtype=np.int32)
+        handle = _vp()
+        _check(_lib.sw_telemetry_create(ne.ctypes.data_as(C.POINTER(_i32)), len(ne), ce.ctypes.data_as(C.POINTER(_i32)),
+                                        len(ce), window, C.byref(handle)), "sw_telemetry_create")
+        self.handle = handle
+
+    def record(self, n: int, c: int, predicted_ns: int, observed_ns: int, slack_ns: int = 0, fallback: bool = False) -> None:
+        _check(_lib.sw_telemetry_record(self.handle, n, c, predicted_ns, observed_ns, slack_ns, int(fallback)),
+               "sw_telemetry_record")
+
+    def margin(self, n: int, c: int, percentile_ppm: int = 990_000, min_samples: int = 1, floor_ns: int = 0) -> int:
+        out = _i64(0)
+        _check(_lib.sw_telemetry_margin(self.handle, n, c, percentile_ppm, min_samples, floor_ns, C.byref(out)),
+               "sw_telemetry_margin")
+        return int(out.value)
+
+    def exceeds(self, n: int, c: int, configured_margin_ns: int, percentile_ppm: int = 990_000, min_samples: int = 1) -> bool:
+        out = _i32(0)
+        _check(_lib.sw_telemetry_exceeds(self.handle, n, c, percentile_ppm, min_samples, configured_margin_ns,
+                                         C.byref(out)), "sw_telemetry_exceeds")
+        return bool(out.value)
+
+    def totals(self) -> dict:
+        t = sw_telemetry_totals()
+        _check(_lib.sw_telemetry_get_totals(self.handle, C.byref(t)), "sw_telemetry_get_totals")
+        return {k: int(getattr(t, k)) for k, _ in t._fields_}
+
+    def close(self):
+        if getattr(self, "handle", None) and _lib is not None:
+            _lib.sw_telemetry_destroy(self.handle)
             self.handle = None
 
     def __del__(self):

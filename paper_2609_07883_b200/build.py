@@ -10,7 +10,7 @@ HERE = Path(__file__).resolve().parent
 CSRC = HERE / "csrc"
 INCLUDE = HERE.parent / "include"
 LIB = HERE / "libsloweave.so"
-SOURCES = ["sw_error.cpp", "sw_controller.cpp", "sw_api.cu", "sw_kernels.cu", "sw_static.cu"]
+SOURCES = ["sw_error.cpp", "sw_controller.cpp", "sw_telemetry.cpp", "sw_api.cu", "sw_kernels.cu", "sw_static.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 

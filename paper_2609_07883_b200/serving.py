@@ -87,12 +87,19 @@ def gpu_executor(ctx, pools, shape: W.AttnShape, c_max: int, max_decode: int, se
 def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, num_pages: int, policy: str = "sloweave",
               c_max: int = 4096, margin_ppm: int = 50_000, margin_abs_ns: int = 0, quantum: int = 16, max_decode: int = 512,
               ctx_cap: int | None = None, seed: int = W.SEED_BASE + 44, log=None, page_tables: bool = True,
-              ttft_slo_ms: float | None = None) -> dict:
+              ttft_slo_ms: float | None = None, telemetry=None, fallback_margin_ns: int | None = None,
+              residual_percentile_ppm: int = 990_000, residual_min_samples: int = 8, fallback_hold: int = 8) -> dict:
     """Run the whole trace; returns statistics.  ``policy`` is "sloweave" or "fixed:<chunk>".  ``execute(batch)`` runs
     one iteration and returns its duration in ns (``gpu_executor`` for the CUDA path).  ``ctx_cap`` clamps the total
     context passed to the table lookup to the table's last grid point.  ``page_tables=False`` hands ``execute`` a batch
     without page lists (enough for a cost model that looks only at sizes; the simulator study runs that way).  With
-    ``ttft_slo_ms`` the result also counts the requests that meet both SLOs and the goodput (Sec. 4.3)."""
+    ``ttft_slo_ms`` the result also counts the requests that meet both SLOs and the goodput (Sec. 4.3).
+
+    ``telemetry`` (a ``binding.Telemetry``) closes the feedback loop of Sec. 3.3 / Sec. 5.1: every iteration's raw table
+    prediction and measured duration are recorded, the residual table's margin for (n, L) is added to the controller's
+    margin, and, when ``fallback_margin_ns`` is given and the residuals exceed it, the iteration runs decode-only.  So
+    that a stale residual cannot starve the queue, at most ``fallback_hold`` consecutive iterations fall back; the next
+    one admits a chunk again under the residual margin and so refreshes the residuals."""
     from . import binding as B
 
     S = shape.page_size
@@ -108,6 +115,7 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
     iters = chunk_iters = 0
     misses_chunk = misses_decode_only = infeasible_flags = stalled_for_memory = 0
     chunks, iter_ns, pred_err = [], [], []
+    fallback_iters = fallback_run = 0
     prefill_tokens = 0
     wall0 = time.time()
     while done < len(reqs):
@@ -136,19 +144,33 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
         budget = int(deadlines.min() - now) if n else 0
         predicted = 0
         flags = 0
-        if fixed_chunk is not None:
+        fell_back = False
+        extra_margin = 0
+        if telemetry is not None and fixed_chunk is None and n and remaining:
+            L_now = min(c_max, remaining)
+            extra_margin = telemetry.margin(n, L_now, residual_percentile_ppm, residual_min_samples, 0)
+            if fallback_margin_ns is not None and fallback_run < fallback_hold and \
+                    telemetry.exceeds(n, L_now, fallback_margin_ns, residual_percentile_ppm, residual_min_samples):
+                fell_back = True
+        if fell_back:
+            c = 0
+            fallback_run += 1
+            fallback_iters += 1
+        elif fixed_chunk is not None:
             c = min(fixed_chunk, remaining)
         else:
             q_eff = quantum if remaining >= quantum else 1   # the last few tokens of a prompt are below the quantum
             prefilled = head.prefilled if head else 0
+            fallback_run = 0
+            m_abs = margin_abs_ns + extra_margin
             ch = B.sw_choose_chunk(table if n else None, now, deadlines, total_ctx, prefilled, remaining,
-                                   c_max=c_max, chunk_quantum=q_eff, margin_abs_ns=margin_abs_ns, margin_ppm=margin_ppm)
+                                   c_max=c_max, chunk_quantum=q_eff, margin_abs_ns=m_abs, margin_ppm=margin_ppm)
             L = min(c_max, remaining)
             if q_eff > 1 and L % q_eff and ch.chunk == L - L % q_eff:
                 # The quantum stopped just short of L.  If L itself fits the budget, take it: a prompt's last few tokens
                 # would otherwise cost a whole extra iteration.
                 fine = B.sw_choose_chunk(table if n else None, now, deadlines, total_ctx, prefilled, remaining, c_max=c_max,
-                                         chunk_quantum=1, margin_abs_ns=margin_abs_ns, margin_ppm=margin_ppm)
+                                         chunk_quantum=1, margin_abs_ns=m_abs, margin_ppm=margin_ppm)
                 if fine.chunk == L:
                     ch = fine
             c, flags, predicted = ch.chunk, ch.flags, ch.predicted_ns
@@ -185,6 +207,9 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
             infeasible_flags += 1
         if predicted and n:
             pred_err.append(dt - predicted)
+        if telemetry is not None and n:
+            raw = table.lookup(n, total_ctx, P, c)      # the table's own prediction, without any margin
+            telemetry.record(n, c, raw, dt, slack_ns=budget - dt, fallback=fell_back)
         still = []
         for r in active:
             r.generated += 1
@@ -239,6 +264,7 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
         "tpot_ms_p99_of_request_p99": float(np.percentile(p99_gap, 99)),
         "requests_meeting_tpot": int(np.sum(p99_gap <= tpot_ms)),
         "prediction_error_ms_p99": float(np.percentile(pred_err, 99)) / MS if pred_err else 0.0,
+        "fallback_iterations": fallback_iters,
         "margin_ppm": margin_ppm, "c_max": c_max, "quantum": quantum, "wall_s": time.time() - wall0,
     }
 
