@@ -38,8 +38,10 @@ def test_binding_lists_the_same_functions(lib_path):
 
     assert sorted(binding.EXPORTS) == declared_functions()
     for name in binding.EXPORTS:
-        assert hasattr(binding, name) or name in ("sw_create", "sw_destroy", "sw_cost_table_create",
-                                                  "sw_cost_table_destroy", "sw_cost_table_lookup")
+        # handles are wrapped by classes (Context, CostTable, Telemetry); everything else has a function of the same name
+        assert hasattr(binding, name) or name.startswith("sw_telemetry_") or name in (
+            "sw_create", "sw_destroy", "sw_cost_table_create", "sw_cost_table_destroy", "sw_cost_table_lookup")
+    assert all(hasattr(binding, cls) for cls in ("Context", "CostTable", "Telemetry"))
 
 
 def test_host_side_argument_errors_without_a_gpu(lib_path):
