@@ -44,7 +44,7 @@ WsLayout ws_layout(const sw_layout& l, int max_chunk, int max_decode, int64_t ma
     w.max_items = sw::kTargetItems + max_decode * l.num_kv_heads;
     size_t off = 0;
     w.ctrl = off;     off = align_up(off + sw::kCtrWords * 4, 256);
-    w.tickets = off;  off = align_up(off + (size_t)std::max(1, max_decode) * l.num_kv_heads * 4, 256);
+    w.tickets = off;  off = align_up(off + (size_t)std::max(1, max_decode) * l.num_kv_heads * 4 * 2, 256);  // tickets, ready
     w.part_ml = off;  off = align_up(off + (size_t)w.max_items * 2 * sw::kMaxGroup * 4, 256);
     w.part_o = off;   off = align_up(off + (size_t)w.max_items * g * l.head_dim * 4, 256);
     const size_t groups = ((size_t)max_chunk + (256 / g) - 1) / (256 / g);
@@ -260,6 +260,7 @@ sw_status run_mixed(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const voi
     }
     p.ctrl = reinterpret_cast<int32_t*>(ctx->ws + ctx->w.ctrl);
     p.tickets = reinterpret_cast<int32_t*>(ctx->ws + ctx->w.tickets);
+    p.ready = p.tickets + (size_t)std::max(1, ctx->max_decode) * l.num_kv_heads;
     p.part_ml = reinterpret_cast<float*>(ctx->ws + ctx->w.part_ml);
     p.part_o = reinterpret_cast<float*>(ctx->ws + ctx->w.part_o);
     p.max_items = ctx->w.max_items;

@@ -50,7 +50,8 @@ struct MixedParams {
     __nv_bfloat16* pool;
     // scratch
     int32_t* ctrl;
-    int32_t* tickets;   // [max_decode * Hkv]
+    int32_t* tickets;   // [max_decode * Hkv]: order in which the units of a (request, kv head) near their end
+    int32_t* ready;     // [max_decode * Hkv]: how many of them have published their partial result
     float* part_ml;     // [max_items][2 * kMaxGroup]  (m then l per query head of the group)
     float* part_o;      // [max_items][group * D]
     int max_items;      // partial-result slots available

@@ -542,11 +542,17 @@ __device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const
     for (int k = 0; k < kStages && k < npg; ++k) issue_next();
     // Once this unit's last page is on its way the following unit is claimed from the shared counter: the counter's
     // round trip hides behind the last pages, and no warp hoards a unit while others are still idle.
+    // With the claim the unit draws its ticket among the units of its (request, kv head): the last ticket makes it
+    // the one that merges.  Both answers are read at the end of the unit, when they have long arrived.
     bool claimed = false;
+    int ticket = 0;  // lane 0
     auto claim_next = [&]() {
         if (!claimed && issued >= npg) {
             claimed = true;
-            if (lane == 0) next_item = pulls ? fixed_items + atomicAdd(&p.ctrl[kCtrWork], 1) : 0x7fffffff;
+            if (lane == 0) {
+                next_item = pulls ? fixed_items + atomicAdd(&p.ctrl[kCtrWork], 1) : 0x7fffffff;
+                if (u.nsplit > 1) ticket = atomicAdd(&p.tickets[u.ticket], 1);
+            }
         }
     };
     claim_next();
@@ -667,7 +673,10 @@ __device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const
         return true;
     }
 
-    // partial result -> scratch, then ticket; the last arriver merges
+    // Partial result -> scratch.  The units that did not draw the last ticket publish it (fence, then one more on the
+    // `ready` counter, without waiting for anything); the one that did waits until the others have and merges.  It is
+    // usually the last to finish, so its wait is short, and no fence or ticket round trip sits between its last page
+    // and the merge.
     if (row_ok) {
         float* po = p.part_o + ((int64_t)u.slot * g + qrow_in_group) * D + (lane & 3) * 2;
 #pragma unroll
@@ -677,16 +686,33 @@ __device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const
             p.part_ml[(int64_t)u.slot * (2 * kMaxGroup) + kMaxGroup + qrow_in_group] = l_run;
         }
     }
-    __threadfence();
-    __syncwarp();
-    int prev = 0;
-    if (lane == 0) prev = atomicAdd(&p.tickets[u.ticket], 1);
-    prev = __shfl_sync(0xffffffffu, prev, 0);
-    if (prev != u.nsplit - 1) return true;
-
-    // last arriver: merge all splits of this (request, kv head)
-    __threadfence();
-    if (lane == 0) p.tickets[u.ticket] = 0;  // ready for the next launch
+    const bool merger = __shfl_sync(0xffffffffu, ticket, 0) == u.nsplit - 1;
+    if (!merger) {
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) atomicAdd(&p.ready[u.ticket], 1);
+        return true;
+    }
+    // last ticket: merge all splits of this (request, kv head) once the others are published
+    __syncwarp();  // this warp's own partial result, written above by all lanes, is ordered before the loads below
+    int ok = 1;
+    if (lane == 0) {
+        const long long t0 = clock64();
+        while (ld_acquire_gpu(&p.ready[u.ticket]) < u.nsplit - 1) {
+            if (clock64() - t0 > kWaitBudgetCycles) {
+                ok = 0;
+                break;
+            }
+            __nanosleep(64);
+        }
+        p.tickets[u.ticket] = 0;  // ready for the next launch
+        p.ready[u.ticket] = 0;
+    }
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    if (!ok) {
+        if (lane == 0) report(p.ctrl, SW_ERR_DEVICE_TIMEOUT, kSiteWait, u.q_row);
+        return false;
+    }
     switch (g) {
         case 1: merge_splits<D, 1>(p, u); break;
         case 2: merge_splits<D, 2>(p, u); break;

@@ -24,7 +24,7 @@ constexpr size_t kPartOBytesPerItem = 4096;              // group * head_dim * 4
 
 constexpr size_t kOffCtrl = 0;
 constexpr size_t kOffTickets = 256;
-constexpr size_t kOffPartMl = kOffTickets + (size_t)kStaticMaxDecode * kStaticMaxKvHeads * 4;
+constexpr size_t kOffPartMl = kOffTickets + (size_t)kStaticMaxDecode * kStaticMaxKvHeads * 4 * 2;  // tickets, ready
 constexpr size_t kOffPartO = kOffPartMl + (size_t)kStaticMaxItems * 2 * sw::kMaxGroup * 4;
 constexpr size_t kScratchBytes = kOffPartO + (size_t)kStaticMaxItems * kPartOBytesPerItem;
 static_assert(kOffPartMl % 256 == 0 && kOffPartO % 256 == 0, "regions stay 256-byte aligned");
@@ -137,6 +137,7 @@ extern "C" sw_status sw_decode_attn_static(const sw_layout* layout, int device, 
     p.lse = lse;
     p.ctrl = reinterpret_cast<int32_t*>(st->scratch + kOffCtrl);
     p.tickets = reinterpret_cast<int32_t*>(st->scratch + kOffTickets);
+    p.ready = p.tickets + kStaticMaxDecode * kStaticMaxKvHeads;
     p.part_ml = reinterpret_cast<float*>(st->scratch + kOffPartMl);
     p.part_o = reinterpret_cast<float*>(st->scratch + kOffPartO);
     p.max_items = kStaticMaxItems;
