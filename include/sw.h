@@ -127,6 +127,13 @@ sw_status sw_cost_probe(sw_ctx* ctx, void* const* kv_pools, int32_t layers, cons
                         void* out, int32_t warmup, int32_t reps, int64_t* p50_ns, int64_t* p99_ns,
                         int64_t* samples_ns, void* stream);
 
+/* The same measurement for a runtime whose iteration is sw_mixed_iteration_run: every timed launch also appends
+ * k_new / v_new (device bf16 [C+n][num_kv_heads][head_dim]) to its pool, so the table holds the cost of what the
+ * executor really launches.  The probed pools are written at the batch's append positions. */
+sw_status sw_cost_probe_iteration(sw_ctx* ctx, void* const* kv_pools, int32_t layers, const sw_batch* batch,
+                                  const void* k_new, const void* v_new, const void* q, void* out, int32_t warmup,
+                                  int32_t reps, int64_t* p50_ns, int64_t* p99_ns, int64_t* samples_ns, void* stream);
+
 /* (No counterpart in the paper.)  Decode-only attention for callers that cannot allocate device memory at all — for
  * example a plugin or a real-time serving loop that runs inside someone else's memory pool, where cudaMalloc is
  * forbidden or would synchronise the device, so neither a context nor a workspace can be created.  It computes what

@@ -53,7 +53,7 @@ class sw_telemetry_totals(C.Structure):
 
 
 EXPORTS = ["sw_workspace_bytes", "sw_create", "sw_destroy", "sw_kv_append", "sw_mixed_attn_run", "sw_mixed_iteration_run",
-           "sw_mixed_iteration_host", "sw_cost_probe", "sw_check_status", "sw_cost_table_create",
+           "sw_mixed_iteration_host", "sw_cost_probe", "sw_cost_probe_iteration", "sw_check_status", "sw_cost_table_create",
            "sw_cost_table_destroy", "sw_cost_table_lookup", "sw_choose_chunk", "sw_last_error",
            "sw_decode_attn_static", "sw_selftest_wait_timeout", "sw_telemetry_create", "sw_telemetry_destroy",
            "sw_telemetry_record", "sw_telemetry_margin", "sw_telemetry_exceeds", "sw_telemetry_get_totals"]
@@ -70,6 +70,8 @@ _lib.sw_mixed_iteration_run.argtypes = [_vp, _vp, C.POINTER(sw_batch), _vp, _vp,
 _lib.sw_mixed_iteration_host.argtypes = [_vp, _vp, C.POINTER(sw_batch), _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.sw_cost_probe.argtypes = [_vp, C.POINTER(_vp), _i32, C.POINTER(sw_batch), _vp, _vp, _i32, _i32,
                                C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), _vp]
+_lib.sw_cost_probe_iteration.argtypes = [_vp, C.POINTER(_vp), _i32, C.POINTER(sw_batch), _vp, _vp, _vp, _vp, _i32, _i32,
+                                         C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), _vp]
 _lib.sw_decode_attn_static.argtypes = [C.POINTER(sw_layout), C.c_int, _vp, C.POINTER(sw_batch), _vp, _vp, _vp, _vp]
 _lib.sw_selftest_wait_timeout.argtypes = [_vp, _i64, _vp]
 _lib.sw_check_status.argtypes = [_vp, _vp, C.POINTER(_i32), C.POINTER(_i32)]
@@ -208,6 +210,20 @@ def sw_mixed_iteration_host(ctx: Context, kv_pool, host_struct: sw_batch, h_q, h
     _check(_lib.sw_mixed_iteration_host(ctx.handle, _ptr(kv_pool), C.byref(host_struct), _ptr(h_q), _ptr(h_k_new),
                                         _ptr(h_v_new), _ptr(h_out), _ptr(h_lse), _stream_handle(stream)),
            "sw_mixed_iteration_host")
+
+
+def sw_cost_probe_iteration(ctx: Context, kv_pools, batch: DeviceBatch, k_new, v_new, q, out, warmup: int = 3,
+                            reps: int = 30, stream=None):
+    """As ``sw_cost_probe`` with the KV append fused into every timed launch."""
+    layers = len(kv_pools)
+    arr = (_vp * layers)(*[_ptr(p) for p in kv_pools])
+    p50, p99 = _i64(0), _i64(0)
+    samples = np.zeros(reps, dtype=np.int64)
+    _check(_lib.sw_cost_probe_iteration(ctx.handle, arr, layers, C.byref(batch.struct), _ptr(k_new), _ptr(v_new), _ptr(q),
+                                        _ptr(out), warmup, reps, C.byref(p50), C.byref(p99),
+                                        samples.ctypes.data_as(C.POINTER(_i64)), _stream_handle(stream)),
+           "sw_cost_probe_iteration")
+    return int(p50.value), int(p99.value), samples
 
 
 def sw_cost_probe(ctx: Context, kv_pools, batch: DeviceBatch, q, out, warmup: int = 3, reps: int = 30, stream=None):

@@ -351,10 +351,13 @@ sw_status sw_mixed_iteration_host(sw_ctx* ctx, void* kv_pool, const sw_batch* hb
     return SW_OK;
 }
 
-sw_status sw_cost_probe(sw_ctx* ctx, void* const* kv_pools, int32_t layers, const sw_batch* batch, const void* q, void* out,
-                        int32_t warmup, int32_t reps, int64_t* p50_ns, int64_t* p99_ns, int64_t* samples_ns, void* stream) {
+namespace {
+// Times iterations of `layers` launches each: attention alone, or (k_new / v_new given) append + attention in one launch.
+sw_status probe(sw_ctx* ctx, void* const* kv_pools, int32_t layers, const sw_batch* batch, const void* k_new,
+                const void* v_new, const void* q, void* out, int32_t warmup, int32_t reps, int64_t* p50_ns, int64_t* p99_ns,
+                int64_t* samples_ns, void* stream, const char* who) {
     if (!ctx || !kv_pools || layers < 1 || reps < 1 || warmup < 0 || !p50_ns || !p99_ns)
-        return sw_fail(SW_ERR_INVALID_ARG, "sw_cost_probe: invalid argument");
+        return sw_fail(SW_ERR_INVALID_ARG, "%s: invalid argument", who);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (!ctx->ev0) SW_CUDA(cudaEventCreate(&ctx->ev0));
     if (!ctx->ev1) SW_CUDA(cudaEventCreate(&ctx->ev1));
@@ -362,7 +365,7 @@ sw_status sw_cost_probe(sw_ctx* ctx, void* const* kv_pools, int32_t layers, cons
     for (int r = -warmup; r < reps; ++r) {
         SW_CUDA(cudaEventRecord(ctx->ev0, s));
         for (int layer = 0; layer < layers; ++layer) {
-            sw_status st = sw_mixed_attn_run(ctx, kv_pools[layer], batch, q, out, nullptr, stream);
+            sw_status st = run_mixed(ctx, kv_pools[layer], batch, k_new, v_new, q, out, nullptr, stream, who);
             if (st != SW_OK) return st;
         }
         SW_CUDA(cudaEventRecord(ctx->ev1, s));
@@ -378,6 +381,21 @@ sw_status sw_cost_probe(sw_ctx* ctx, void* const* kv_pools, int32_t layers, cons
     *p50_ns = rank(0.50);
     *p99_ns = rank(0.99);
     return SW_OK;
+}
+}  // namespace
+
+sw_status sw_cost_probe(sw_ctx* ctx, void* const* kv_pools, int32_t layers, const sw_batch* batch, const void* q, void* out,
+                        int32_t warmup, int32_t reps, int64_t* p50_ns, int64_t* p99_ns, int64_t* samples_ns, void* stream) {
+    return probe(ctx, kv_pools, layers, batch, nullptr, nullptr, q, out, warmup, reps, p50_ns, p99_ns, samples_ns, stream,
+                 "sw_cost_probe");
+}
+
+sw_status sw_cost_probe_iteration(sw_ctx* ctx, void* const* kv_pools, int32_t layers, const sw_batch* batch, const void* k_new,
+                                  const void* v_new, const void* q, void* out, int32_t warmup, int32_t reps, int64_t* p50_ns,
+                                  int64_t* p99_ns, int64_t* samples_ns, void* stream) {
+    if (!k_new || !v_new) return sw_fail(SW_ERR_INVALID_ARG, "sw_cost_probe_iteration: null tensor");
+    return probe(ctx, kv_pools, layers, batch, k_new, v_new, q, out, warmup, reps, p50_ns, p99_ns, samples_ns, stream,
+                 "sw_cost_probe_iteration");
 }
 
 sw_status sw_check_status(sw_ctx* ctx, void* stream, int32_t* code, int32_t* detail) {

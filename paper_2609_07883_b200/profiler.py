@@ -36,8 +36,8 @@ def pages_needed(shape: W.AttnShape, n: int, ctx_total: int, prefix: int, chunk:
 
 
 def measure_table(ctx, pools, shape: W.AttnShape, num_pages: int, n_grid, ctx_grid, prefix_grid, chunk_grid,
-                  reps: int = 10, warmup: int = 2, seed: int = W.SEED_BASE + 40, progress=None) -> dict:
-    """Probe every grid point.  ``ctx`` is a binding.Context big enough for the largest point; ``pools`` the layer
+                  reps: int = 10, warmup: int = 2, seed: int = W.SEED_BASE + 40, progress=None, fused: bool = False) -> dict:
+    """Probe every grid point (``fused``: with the KV append in every launch, as ``sw_mixed_iteration_run`` runs it).  ``ctx`` is a binding.Context big enough for the largest point; ``pools`` the layer
     stack (list of device tensors).  Returns a plain dict (JSON-serialisable) with P50 and P99 per point."""
     import torch
 
@@ -50,6 +50,10 @@ def measure_table(ctx, pools, shape: W.AttnShape, num_pages: int, n_grid, ctx_gr
     gen.manual_seed(seed)
     q = torch.randn(max_rows, shape.num_q_heads, shape.head_dim, device=dev, generator=gen).to(torch.bfloat16)
     out = torch.empty_like(q)
+    k_new = v_new = None
+    if fused:
+        k_new = torch.randn(max_rows, shape.num_kv_heads, shape.head_dim, device=dev, generator=gen).to(torch.bfloat16)
+        v_new = torch.randn(max_rows, shape.num_kv_heads, shape.head_dim, device=dev, generator=gen).to(torch.bfloat16)
     shape4 = (len(n_grid), len(ctx_grid), len(prefix_grid), len(chunk_grid))
     p50 = np.zeros(shape4, dtype=np.int64)
     p99 = np.zeros(shape4, dtype=np.int64)
@@ -65,14 +69,17 @@ def measure_table(ctx, pools, shape: W.AttnShape, num_pages: int, n_grid, ctx_gr
                         continue
                     batch = probe_batch(shape, num_pages, int(n), int(ctx_total), int(prefix), int(chunk), rng)
                     db = B.DeviceBatch(batch, dev)
-                    m, h, _ = B.sw_cost_probe(ctx, pools, db, q, out, warmup=warmup, reps=reps)
+                    if fused:
+                        m, h, _ = B.sw_cost_probe_iteration(ctx, pools, db, k_new, v_new, q, out, warmup=warmup, reps=reps)
+                    else:
+                        m, h, _ = B.sw_cost_probe(ctx, pools, db, q, out, warmup=warmup, reps=reps)
                     p50[a, b, c_i, e], p99[a, b, c_i, e] = m, h
         if progress:
             progress(f"n={n}: {time.time() - t0:.1f}s")
     B.sw_check_status(ctx)
     return {"n_grid": [int(x) for x in n_grid], "ctx_grid": [int(x) for x in ctx_grid],
             "prefix_grid": [int(x) for x in prefix_grid], "chunk_grid": [int(x) for x in chunk_grid],
-            "layers": len(pools), "reps": reps, "warmup": warmup, "p50_ns": p50.tolist(), "p99_ns": p99.tolist(),
+            "layers": len(pools), "reps": reps, "warmup": warmup, "fused_append": bool(fused), "p50_ns": p50.tolist(), "p99_ns": p99.tolist(),
             "shape": [shape.num_q_heads, shape.num_kv_heads, shape.head_dim, shape.page_size]}
 
 

@@ -313,7 +313,7 @@ def main(argv=None):
         ctx_grid = [t for t in (8192, 65536, 196608, 393216) if t < ctx_top] + [ctx_top]
         log(f"measuring cost table: {len(n_grid) * len(ctx_grid) * len(prefix_grid) * len(chunk_grid)} points, {args.layers} layers")
         tab = profiler.measure_table(ctx, pools, shape, args.pages, n_grid, ctx_grid, prefix_grid, chunk_grid,
-                                     reps=args.table_reps, warmup=2, progress=log)
+                                     reps=args.table_reps, warmup=2, progress=log, fused=True)
         if args.table:
             profiler.save_table(tab, args.table)
     table = profiler.to_cost_table(tab)

@@ -42,6 +42,17 @@ def test_cost_probe_returns_ordered_percentiles(setup):
     assert samples.min() <= p50 <= p99 <= samples.max()
     assert p50 == np.sort(samples)[9] and p99 == np.sort(samples)[19]   # nearest rank: ceil(q * reps)-th smallest
     assert B.sw_check_status(ctx, raise_on_error=False) == (0, 0)
+    # the probe of the fused launch appends the rows to every probed pool and costs about the same
+    k_new = torch.randn(batch.num_rows, shape.num_kv_heads, shape.head_dim, device=pools[0].device).to(torch.bfloat16)
+    v_new = torch.randn_like(k_new)
+    f50, f99, fs = B.sw_cost_probe_iteration(ctx, pools, db, k_new, v_new, q, out, warmup=2, reps=20)
+    assert fs.min() > 0 and fs.min() <= f50 <= f99 <= fs.max()
+    assert 0.5 * p50 < f50 < 2.0 * p50
+    page, slot = int(batch.decode_pages[batch.decode_page_indptr[1] + (300 - 1) // 16]), (300 - 1) % 16
+    for pool in pools:
+        row = pool.view(pages, 2, shape.num_kv_heads, 16, shape.head_dim)[page, 0, :, slot, :]
+        assert torch.equal(row, k_new[batch.chunk_len + 1])           # request 1 (length 300): its new K row
+    assert B.sw_check_status(ctx, raise_on_error=False) == (0, 0)
 
 
 def test_measured_table_is_made_monotone_and_drives_the_loop(setup):
@@ -49,7 +60,8 @@ def test_measured_table_is_made_monotone_and_drives_the_loop(setup):
     from paper_2609_07883_b200 import profiler, serving
 
     n_grid, ctx_grid, prefix_grid, chunk_grid = [1, 8, 64], [2048, 30000], [0, 4096], [0, 64, 256, 512]
-    tab = profiler.measure_table(ctx, pools, shape, pages, n_grid, ctx_grid, prefix_grid, chunk_grid, reps=4, warmup=1)
+    tab = profiler.measure_table(ctx, pools, shape, pages, n_grid, ctx_grid, prefix_grid, chunk_grid, reps=4, warmup=1,
+                                 fused=True)
     raw = np.asarray(tab["p99_ns"])
     assert raw.shape == (3, 2, 2, 4) and (raw > 0).all()
     table = profiler.to_cost_table(tab)
