@@ -192,11 +192,14 @@ def reduce_max_over_ranks(x: float, device=None) -> float:
     return float(t.item())
 
 
-def aggregate_result(per_rank_us: float, world: int, chunk: int, decodes: int, device=None) -> dict:
-    """Whole-job numbers of N independent replicas: the iteration time is the slowest rank's, throughputs add up."""
+def aggregate_result(per_rank_us: float, world: int, chunk: int, decodes: int, device=None, sharded: bool = False) -> dict:
+    """Whole-job numbers.  N independent replicas: the iteration time is the slowest rank's, throughputs add up.  One
+    iteration sharded by KV heads over N ranks (``sharded``): the iteration ends with its slowest rank and there is still
+    one iteration's worth of tokens."""
     us = reduce_max_over_ranks(per_rank_us, device)
-    return {"value": us, "iterations_per_s": world / (us * 1e-6), "prefill_tokens_per_s": world * chunk / (us * 1e-6),
-            "decode_tokens_per_s": world * decodes / (us * 1e-6)}
+    jobs = 1 if sharded else world
+    return {"value": us, "iterations_per_s": jobs / (us * 1e-6), "prefill_tokens_per_s": jobs * chunk / (us * 1e-6),
+            "decode_tokens_per_s": jobs * decodes / (us * 1e-6)}
 
 
 # ---------------------------------------------------------------------------------------------------------------
@@ -251,7 +254,13 @@ def run_ours(args) -> dict:
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    batch = make_workload(args, rank)
+    sharded = args.parallel == "heads" and world > 1
+    batch = make_workload(args, 0 if sharded else rank)
+    if sharded:
+        # every rank runs the same iteration on its share of the KV heads (and of the query heads that read them)
+        from paper_2609_07883_b200 import sharding
+
+        batch = sharding.shard_batch(batch, world)
     sh = batch.shape
     work = attention_work(batch)
     total_pages = int(batch.prefill_pages.shape[0] + batch.decode_pages.shape[0])
@@ -301,7 +310,7 @@ def run_ours(args) -> dict:
     e1.record()
     sync_all()
     ms_local = e0.elapsed_time(e1)
-    agg = aggregate_result(ms_local / args.steps * 1e3, world, batch.chunk_len, batch.num_decode, dev)
+    agg = aggregate_result(ms_local / args.steps * 1e3, world, batch.chunk_len, batch.num_decode, dev, sharded)
     ms_total = agg["value"] * args.steps / 1e3
     # (2) the attention launch alone (dominant kernel) for the roofline, same stream, same rotation
     a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -347,7 +356,8 @@ def run_ours(args) -> dict:
     traffic = NCU_TRAFFIC_DEFAULT_WORKLOAD if is_default else None
     result = {
         "metric": "mixed_iteration_us", "value": us, "unit": "us", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": False, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": False,
+        "scaling": "strong" if sharded else "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(args, batch),
         "iterations_per_s": agg["iterations_per_s"],
         "prefill_tokens_per_s": agg["prefill_tokens_per_s"],
@@ -387,6 +397,8 @@ def main():
     ap.add_argument("--cpu-budget-keys", type=int, default=1_000_000_000)
     ap.add_argument("--ref-budget-keys", type=int, default=1_000_000_000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--parallel", default="replicas", choices=["replicas", "heads"],
+                    help="N > 1: independent replicas (default) or one iteration sharded by KV heads, no collective either way")
     args = ap.parse_args()
     dn, dc, dp = WORKLOAD_DEFAULTS[args.workload]
     args.decodes = dn if args.decodes is None else args.decodes

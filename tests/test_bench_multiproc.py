@@ -23,6 +23,7 @@ def _worker(rank, world, port, out_dir):
     assert bench.dist_env() == (rank, rank, world)
     per_rank_us = 100.0 + 50.0 * rank            # rank 1 is the slow one
     agg = bench.aggregate_result(per_rank_us, world, chunk=512, decodes=64)
+    agg["sharded"] = bench.aggregate_result(per_rank_us, world, chunk=512, decodes=64, sharded=True)
     dist.barrier()
     Path(out_dir, f"rank{rank}.json").write_text(json.dumps(agg))
     dist.destroy_process_group()
@@ -37,6 +38,10 @@ def test_two_gloo_ranks_take_the_max_and_add_throughputs(tmp_path):
         assert abs(agg["iterations_per_s"] - 2 / 150e-6) < 1e-6        # two replicas finish one iteration each
         assert abs(agg["prefill_tokens_per_s"] - 2 * 512 / 150e-6) < 1e-3
         assert abs(agg["decode_tokens_per_s"] - 2 * 64 / 150e-6) < 1e-3
+        # one iteration sharded by KV heads over the two ranks: still the slowest rank, but one iteration's tokens
+        sh = agg["sharded"]
+        assert sh["value"] == 150.0 and abs(sh["iterations_per_s"] - 1 / 150e-6) < 1e-6
+        assert abs(sh["prefill_tokens_per_s"] - 512 / 150e-6) < 1e-3
 
 
 def test_single_process_is_the_identity():
