@@ -66,7 +66,19 @@ typedef struct {
     const int32_t* decode_kv_len;     /* [n] keys attended by request i, INCLUDING the token appended now */
     const int32_t* decode_page_indptr;/* [n+1] CSR offsets into decode_pages */
     const int32_t* decode_pages;      /* [indptr[n]] page ids */
+    /* Several prefill chunks in one iteration (Sec. 3.3, "Prefill batching"): with num_chunks > 0 the three arrays
+     * below, which are HOST arrays, replace prefix_len / chunk_len.  Chunk j has chunk_lens[j] tokens at prefix
+     * chunk_prefix_lens[j] of its own prompt; its rows follow those of chunk j-1 in q / k_new / v_new / out (C is then
+     * the sum of the chunk lengths), and its prompt's page list is
+     * prefill_pages[chunk_page_indptr[j] .. chunk_page_indptr[j+1]) with chunk_page_indptr[num_chunks] ==
+     * num_prefill_pages.  At most SW_MAX_CHUNKS chunks; list the longest first (they are scheduled in this order).
+     * num_chunks == 0 (all three pointers ignored) is the single chunk described by prefix_len / chunk_len. */
+    int32_t num_chunks;
+    const int32_t* chunk_prefix_lens;
+    const int32_t* chunk_lens;
+    const int32_t* chunk_page_indptr;
 } sw_batch;
+#define SW_MAX_CHUNKS 8
 
 /* ---- context -------------------------------------------------------------------------------------- */
 

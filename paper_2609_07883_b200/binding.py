@@ -34,7 +34,17 @@ class sw_layout(C.Structure):
 class sw_batch(C.Structure):
     _fields_ = [("prefix_len", C.c_int32), ("chunk_len", C.c_int32), ("prefill_pages", C.c_void_p),
                 ("num_prefill_pages", C.c_int32), ("num_decode", C.c_int32), ("decode_kv_len", C.c_void_p),
-                ("decode_page_indptr", C.c_void_p), ("decode_pages", C.c_void_p)]
+                ("decode_page_indptr", C.c_void_p), ("decode_pages", C.c_void_p), ("num_chunks", C.c_int32),
+                ("chunk_prefix_lens", C.c_void_p), ("chunk_lens", C.c_void_p), ("chunk_page_indptr", C.c_void_p)]
+
+
+def _chunk_fields(batch):
+    """(num_chunks, three HOST pointers, keepalive) of a batch's chunk arrays; zeros for a single-chunk batch."""
+    if getattr(batch, "chunk_lens", None) is None:
+        return 0, None, None, None, []
+    arrs = [np.ascontiguousarray(a, dtype=np.int32) for a in
+            (batch.chunk_prefix_lens, batch.chunk_lens, batch.chunk_page_indptr)]
+    return len(arrs[1]), arrs[0].ctypes.data, arrs[1].ctypes.data, arrs[2].ctypes.data, arrs
 
 
 class sw_chooser_params(C.Structure):
@@ -176,18 +186,20 @@ class DeviceBatch:
         self.decode_kv_len = to(batch.decode_kv_len)
         self.decode_page_indptr = to(batch.decode_page_indptr)
         self.decode_pages = to(batch.decode_pages)
+        nch, cp, cl, ci, self._chunk_keep = _chunk_fields(batch)
         self.struct = sw_batch(batch.prefix_len, batch.chunk_len, self.prefill_pages.data_ptr(),
                                int(self.prefill_pages.numel()), batch.num_decode, self.decode_kv_len.data_ptr(),
-                               self.decode_page_indptr.data_ptr(), self.decode_pages.data_ptr())
+                               self.decode_page_indptr.data_ptr(), self.decode_pages.data_ptr(), nch, cp, cl, ci)
 
 
 def host_batch_struct(batch):
     """``sw_batch`` whose pointers are HOST pointers (for sw_mixed_iteration_host); returns (struct, keepalive)."""
     arrs = [np.ascontiguousarray(a, dtype=np.int32) for a in
             (batch.prefill_pages, batch.decode_kv_len, batch.decode_page_indptr, batch.decode_pages)]
+    nch, cp, cl, ci, keep = _chunk_fields(batch)
     s = sw_batch(batch.prefix_len, batch.chunk_len, arrs[0].ctypes.data, int(arrs[0].shape[0]), batch.num_decode,
-                 arrs[1].ctypes.data, arrs[2].ctypes.data, arrs[3].ctypes.data)
-    return s, arrs
+                 arrs[1].ctypes.data, arrs[2].ctypes.data, arrs[3].ctypes.data, nch, cp, cl, ci)
+    return s, arrs + keep
 
 
 def sw_kv_append(ctx: Context, kv_pool, batch: DeviceBatch, k_new, v_new, stream=None) -> None:

@@ -106,20 +106,72 @@ sw_status kv_map_for(sw_ctx* ctx, const void* pool, const sw::KvMaps** out) {
     return SW_OK;
 }
 
-sw_status check_batch(const sw_ctx* ctx, const sw_batch* b, const char* who) {
+// The prefill chunks of a batch in the form the kernels take (single-chunk batches become one chunk).
+struct Chunks {
+    int n = 0;
+    int rows = 0;  // chunk rows of the iteration = sum of the chunk lengths
+    int P[sw::kMaxChunks] = {}, C[sw::kMaxChunks] = {}, row0[sw::kMaxChunks] = {}, page0[sw::kMaxChunks + 1] = {};
+};
+static_assert(SW_MAX_CHUNKS == sw::kMaxChunks, "the header states the limit");
+
+sw_status chunks_of(const sw_batch* b, const char* who, Chunks* out) {
+    Chunks c;
+    if (b->num_chunks < 0 || b->num_chunks > sw::kMaxChunks)
+        return sw_fail(SW_ERR_INVALID_ARG, "%s: num_chunks %d outside 0..%d", who, b->num_chunks, sw::kMaxChunks);
+    if (b->num_chunks == 0) {
+        if (b->chunk_len > 0) {
+            c.n = 1;
+            c.P[0] = b->prefix_len;
+            c.C[0] = b->chunk_len;
+            c.rows = b->chunk_len;
+            c.page0[1] = b->num_prefill_pages;
+        }
+    } else {
+        if (!b->chunk_prefix_lens || !b->chunk_lens || !b->chunk_page_indptr)
+            return sw_fail(SW_ERR_INVALID_ARG, "%s: chunk arrays missing", who);
+        int64_t rows = 0;
+        for (int j = 0; j < b->num_chunks; ++j) {
+            if (b->chunk_prefix_lens[j] < 0 || b->chunk_lens[j] < 1)
+                return sw_fail(SW_ERR_INVALID_ARG, "%s: chunk %d has prefix %d and length %d", who, j, b->chunk_prefix_lens[j],
+                               b->chunk_lens[j]);
+            if (b->chunk_page_indptr[j + 1] < b->chunk_page_indptr[j] || b->chunk_page_indptr[0] != 0)
+                return sw_fail(SW_ERR_INVALID_ARG, "%s: chunk_page_indptr must start at 0 and not decrease", who);
+            c.P[j] = b->chunk_prefix_lens[j];
+            c.C[j] = b->chunk_lens[j];
+            c.row0[j] = (int)rows;
+            c.page0[j] = b->chunk_page_indptr[j];
+            rows += b->chunk_lens[j];
+            if (rows > sw::kMaxChunk) return sw_fail(SW_ERR_UNSUPPORTED, "%s: more than %d chunk rows", who, sw::kMaxChunk);
+        }
+        c.n = b->num_chunks;
+        c.rows = (int)rows;
+        c.page0[c.n] = b->chunk_page_indptr[c.n];
+        if (c.page0[c.n] != b->num_prefill_pages)
+            return sw_fail(SW_ERR_INVALID_ARG, "%s: chunk_page_indptr ends at %d, num_prefill_pages is %d", who, c.page0[c.n],
+                           b->num_prefill_pages);
+    }
+    for (int j = c.n; j <= sw::kMaxChunks; ++j) c.page0[j] = c.page0[c.n];
+    *out = c;
+    return SW_OK;
+}
+
+sw_status check_batch(const sw_ctx* ctx, const sw_batch* b, const char* who, Chunks* chunks) {
     if (!ctx || !b) return sw_fail(SW_ERR_INVALID_ARG, "%s: null context or batch", who);
     if (b->prefix_len < 0 || b->chunk_len < 0 || b->num_decode < 0 || b->num_prefill_pages < 0)
         return sw_fail(SW_ERR_INVALID_ARG, "%s: negative size in batch", who);
-    if (b->chunk_len > ctx->max_chunk || b->num_decode > ctx->max_decode)
-        return sw_fail(SW_ERR_WORKSPACE, "%s: chunk_len %d / num_decode %d exceed the context's limits %d / %d", who,
-                       b->chunk_len, b->num_decode, ctx->max_chunk, ctx->max_decode);
+    sw_status cs = chunks_of(b, who, chunks);
+    if (cs != SW_OK) return cs;
+    if (chunks->rows > ctx->max_chunk || b->num_decode > ctx->max_decode)
+        return sw_fail(SW_ERR_WORKSPACE, "%s: %d chunk rows / num_decode %d exceed the context's limits %d / %d", who,
+                       chunks->rows, b->num_decode, ctx->max_chunk, ctx->max_decode);
     if (b->num_decode > sw::kMaxDecode)
         return sw_fail(SW_ERR_UNSUPPORTED, "%s: at most %d decode requests per iteration", who, sw::kMaxDecode);
-    if (b->chunk_len > 0) {
-        const int64_t need = ((int64_t)b->prefix_len + b->chunk_len + sw::kPageSize - 1) / sw::kPageSize;
-        if (!b->prefill_pages || b->num_prefill_pages < need)
-            return sw_fail(SW_ERR_OUT_OF_RANGE, "%s: prefill page list has %d entries, P+C needs %lld", who,
-                           b->num_prefill_pages, (long long)need);
+    for (int j = 0; j < chunks->n; ++j) {
+        const int64_t need = ((int64_t)chunks->P[j] + chunks->C[j] + sw::kPageSize - 1) / sw::kPageSize;
+        const int have = chunks->page0[j + 1] - chunks->page0[j];
+        if (!b->prefill_pages || have < need)
+            return sw_fail(SW_ERR_OUT_OF_RANGE, "%s: prefill page list has %d entries, P+C needs %lld", who, have,
+                           (long long)need);
     }
     if (b->num_decode > 0 && (!b->decode_kv_len || !b->decode_page_indptr || !b->decode_pages))
         return sw_fail(SW_ERR_INVALID_ARG, "%s: decode arrays missing", who);
@@ -194,9 +246,10 @@ void sw_destroy(sw_ctx* ctx) {
 
 sw_status sw_kv_append(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const void* k_new, const void* v_new,
                        void* stream) {
-    sw_status st = check_batch(ctx, batch, "sw_kv_append");
+    Chunks ch;
+    sw_status st = check_batch(ctx, batch, "sw_kv_append", &ch);
     if (st != SW_OK) return st;
-    if (batch->chunk_len + batch->num_decode == 0) return SW_OK;
+    if (ch.rows + batch->num_decode == 0) return SW_OK;
     if (!kv_pool || !k_new || !v_new) return sw_fail(SW_ERR_INVALID_ARG, "sw_kv_append: null tensor");
     if (((reinterpret_cast<uintptr_t>(kv_pool) | reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new)) & 15) != 0)
         return sw_fail(SW_ERR_INVALID_ARG, "sw_kv_append: tensors must be 16-byte aligned");
@@ -204,9 +257,13 @@ sw_status sw_kv_append(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const 
     p.Hkv = ctx->layout.num_kv_heads;
     p.D = ctx->layout.head_dim;
     p.num_pages = ctx->layout.num_pages;
-    p.P = batch->prefix_len;
-    p.C = batch->chunk_len;
+    p.C = ch.rows;
     p.n = batch->num_decode;
+    p.nchunks = ch.n;
+    std::memcpy(p.cP, ch.P, sizeof p.cP);
+    std::memcpy(p.cC, ch.C, sizeof p.cC);
+    std::memcpy(p.cRow0, ch.row0, sizeof p.cRow0);
+    std::memcpy(p.cPage0, ch.page0, sizeof p.cPage0);
     p.prefill_pages = batch->prefill_pages;
     p.num_prefill_pages = batch->num_prefill_pages;
     p.decode_kv_len = batch->decode_kv_len;
@@ -224,9 +281,10 @@ namespace {
 // The attention launch; with k_new / v_new non-null the same launch first writes those rows into the pool.
 sw_status run_mixed(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const void* k_new, const void* v_new, const void* q,
                     void* out, float* lse, void* stream, const char* who) {
-    sw_status st = check_batch(ctx, batch, who);
+    Chunks ch;
+    sw_status st = check_batch(ctx, batch, who, &ch);
     if (st != SW_OK) return st;
-    if (batch->chunk_len + batch->num_decode == 0) return SW_OK;
+    if (ch.rows + batch->num_decode == 0) return SW_OK;
     if (!kv_pool || !q || !out) return sw_fail(SW_ERR_INVALID_ARG, "%s: null tensor", who);
     if (((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(k_new) |
           reinterpret_cast<uintptr_t>(v_new)) & 15) != 0)
@@ -242,9 +300,13 @@ sw_status run_mixed(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const voi
     p.num_pages = l.num_pages;
     p.sm_scale = l.sm_scale;
     p.sm_scale_log2 = l.sm_scale * 1.4426950408889634f;
-    p.P = batch->prefix_len;
-    p.C = batch->chunk_len;
+    p.C = ch.rows;
     p.n = batch->num_decode;
+    p.nchunks = ch.n;
+    std::memcpy(p.cP, ch.P, sizeof p.cP);
+    std::memcpy(p.cC, ch.C, sizeof p.cC);
+    std::memcpy(p.cRow0, ch.row0, sizeof p.cRow0);
+    std::memcpy(p.cPage0, ch.page0, sizeof p.cPage0);
     p.prefill_pages = batch->prefill_pages;
     p.num_prefill_pages = batch->num_prefill_pages;
     p.decode_kv_len = batch->decode_kv_len;
@@ -301,10 +363,13 @@ sw_status sw_mixed_iteration_host(sw_ctx* ctx, void* kv_pool, const sw_batch* hb
                                   const void* h_v_new, void* h_out, float* h_lse, void* stream) {
     sw_status st = SW_OK;
     if (!ctx || !hb) return sw_fail(SW_ERR_INVALID_ARG, "sw_mixed_iteration_host: null context or batch");
-    if (hb->chunk_len < 0 || hb->num_decode < 0 || hb->num_prefill_pages < 0 || hb->chunk_len > ctx->max_chunk ||
+    Chunks hch;
+    st = chunks_of(hb, "sw_mixed_iteration_host", &hch);
+    if (st != SW_OK) return st;
+    if (hb->chunk_len < 0 || hb->num_decode < 0 || hb->num_prefill_pages < 0 || hch.rows > ctx->max_chunk ||
         hb->num_decode > ctx->max_decode)
         return sw_fail(SW_ERR_WORKSPACE, "sw_mixed_iteration_host: batch exceeds the context's limits");
-    const int rows = hb->chunk_len + hb->num_decode;
+    const int rows = hch.rows + hb->num_decode;
     if (rows == 0) return SW_OK;
     if (!h_q || !h_k_new || !h_v_new || !h_out || !kv_pool)
         return sw_fail(SW_ERR_INVALID_ARG, "sw_mixed_iteration_host: null tensor");

@@ -17,6 +17,7 @@ constexpr int kTargetItems = 4096;      // split-KV units aimed at per launch (b
 constexpr int kMinSplitTokens = 128;    // never split a decode context finer than this
 constexpr int kMaxGroup = 8;            // query heads per KV head
 constexpr int kMaxCtas = 192;           // persistent CTAs (one per SM) the scratch is sized for
+constexpr int kMaxChunks = 8;           // prefill chunks (of different prompts) in one iteration
 constexpr int kMaxChunk = 65536;        // chunk tokens per iteration (256-row groups are planned in shared memory)
 
 // Control words at the start of the workspace.
@@ -33,8 +34,12 @@ struct MixedParams {
     int64_t num_pages;
     float sm_scale;       // softmax scale
     float sm_scale_log2;  // sm_scale * log2(e)
-    // batch
-    int P, C, n;
+    // batch.  C is the number of chunk rows of the iteration: the rows of its prefill chunks, one chunk after the
+    // other.  Chunk j has cC[j] tokens at prefix cP[j], starts at row cRow0[j] and its prompt's page list starts at
+    // prefill_pages[cPage0[j]] (cPage0[nchunks] = num_prefill_pages).
+    int C, n;
+    int nchunks;
+    int cP[kMaxChunks], cC[kMaxChunks], cRow0[kMaxChunks], cPage0[kMaxChunks + 1];
     const int32_t* prefill_pages;
     int num_prefill_pages;
     const int32_t* decode_kv_len;
@@ -65,7 +70,9 @@ struct MixedParams {
 struct AppendParams {
     int Hkv, D;
     int64_t num_pages;
-    int P, C, n;
+    int C, n;
+    int nchunks;
+    int cP[kMaxChunks], cC[kMaxChunks], cRow0[kMaxChunks], cPage0[kMaxChunks + 1];
     const int32_t* prefill_pages;
     int num_prefill_pages;
     const int32_t* decode_kv_len;

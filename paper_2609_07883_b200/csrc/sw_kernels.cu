@@ -37,9 +37,11 @@ __device__ __forceinline__ void append_rows(const AppendParams& p, int64_t first
         const int32_t* pages;
         int npages;
         if (row < p.C) {
-            pos = (int64_t)p.P + row;
-            pages = p.prefill_pages;
-            npages = p.num_prefill_pages;
+            int j = 0;  // the chunk this row belongs to
+            while (j + 1 < p.nchunks && row >= p.cRow0[j + 1]) ++j;
+            pos = (int64_t)p.cP[j] + (row - p.cRow0[j]);
+            pages = p.prefill_pages + p.cPage0[j];
+            npages = p.cPage0[j + 1] - p.cPage0[j];
         } else {
             const int i = row - p.C;
             const int len = p.decode_kv_len[i];
@@ -769,9 +771,16 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
         a.Hkv = p.Hkv;
         a.D = D;
         a.num_pages = p.num_pages;
-        a.P = p.P;
         a.C = p.C;
         a.n = p.n;
+        a.nchunks = p.nchunks;
+        for (int j = 0; j < kMaxChunks; ++j) {
+            a.cP[j] = p.cP[j];
+            a.cC[j] = p.cC[j];
+            a.cRow0[j] = p.cRow0[j];
+            a.cPage0[j] = p.cPage0[j];
+        }
+        a.cPage0[kMaxChunks] = p.cPage0[kMaxChunks];
         a.prefill_pages = p.prefill_pages;
         a.num_prefill_pages = p.num_prefill_pages;
         a.decode_kv_len = p.decode_kv_len;
@@ -798,7 +807,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
         const PfPlan pplan = pf_make_plan(p);
         prefill_ctas = min(pplan.n_entries, (int)gridDim.x);
         late.ctas = prefill_ctas;
-        late.us = kLateBaseUs + kLateStepUs * ((pf_steps_of_rank(p, pplan.n_tp, 0) + pplan.pieces - 1) / pplan.pieces);
+        late.us = kLateBaseUs + kLateStepUs * ((pplan.longest + pplan.pieces - 1) / pplan.pieces);
         const int first_entry = blockIdx.x;
         if (first_entry < pplan.n_entries) {  // CTA-uniform: this CTA has prefill work
             if (warp == 1) {

@@ -75,8 +75,9 @@ __device__ __forceinline__ bool pf_wait(const PfShared& sh, int bar, uint32_t pa
 constexpr int kPfMinPieceSteps = SW_PF_MIN_PIECE_STEPS;
 
 struct PfPlan {
-    int n_tp;           // 256-row groups of the chunk
-    int n_items;        // n_tp * Hkv
+    int items_before[kMaxChunks + 1];  // items of the chunks before chunk j (items are numbered chunk by chunk)
+    int longest, shortest;             // steps of the longest and of the shortest item
+    int n_items;        // sum over chunks of (256-row groups) * Hkv
     int n_whole;        // entries [0, n_whole) are whole items
     int pieces;         // k: pieces per tail item (1 = tail items are whole too)
     int n_entries;      // n_whole + (n_items - n_whole) * k
@@ -84,8 +85,11 @@ struct PfPlan {
 };
 
 struct PfItem {
-    int item;        // rank * Hkv + kvh
+    int item;        // number of the item among all chunks' items; within its chunk: rank * Hkv + kvh
     int kvh;
+    int P, C;        // the chunk's prefix length and tokens
+    int row0;        // the chunk's first row of q / out
+    const int32_t* pages;  // the page list of the chunk's prompt
     int tok0[2];     // first chunk token of each tile
     int nkv[2];      // KV tiles each tile attends in total (0 = tile has no rows)
     int nk;          // steps of the item = max(nkv)
@@ -94,20 +98,20 @@ struct PfItem {
     int slot0;       // scratch slot of the item's piece 0 (tail items only)
 };
 
-__device__ __forceinline__ int pf_tiles_of(const MixedParams& p, int tok0) {
-    const int tt = 128 / p.group;  // tokens per tile
-    if (tok0 >= p.C) return 0;
-    return (p.P + min(tok0 + tt, p.C) - 1) / 128 + 1;
+__device__ __forceinline__ int pf_tiles_of(int group, int P, int C, int tok0) {
+    const int tt = 128 / group;  // tokens per tile
+    if (tok0 >= C) return 0;
+    return (P + min(tok0 + tt, C) - 1) / 128 + 1;
 }
-__device__ __forceinline__ int pf_num_groups(const MixedParams& p) {
-    const int tok_per_item = 256 / p.group;
-    return (p.C + tok_per_item - 1) / tok_per_item;
+__device__ __forceinline__ int pf_num_groups(int group, int C) {
+    const int tok_per_item = 256 / group;
+    return (C + tok_per_item - 1) / tok_per_item;
 }
-// steps of one item of rank r (the later tile, when it has rows, attends the most keys)
-__device__ __forceinline__ int pf_steps_of_rank(const MixedParams& p, int n_tp, int r) {
-    const int tt = 128 / p.group;
+// steps of one item of rank r of a chunk with n_tp groups (the later tile, when it has rows, attends the most keys)
+__device__ __forceinline__ int pf_steps_of_rank(int group, int P, int C, int n_tp, int r) {
+    const int tt = 128 / group;
     const int tp = n_tp - 1 - r;
-    return max(pf_tiles_of(p, (tp * 2) * tt), pf_tiles_of(p, (tp * 2 + 1) * tt));
+    return max(pf_tiles_of(group, P, C, (tp * 2) * tt), pf_tiles_of(group, P, C, (tp * 2 + 1) * tt));
 }
 // first KV tile of piece i when nk steps are cut into k pieces
 __device__ __forceinline__ int pf_piece_begin(int nk, int k, int i) { return (int)(((long long)nk * i) / k); }
@@ -115,16 +119,30 @@ __device__ __forceinline__ int pf_piece_begin(int nk, int k, int i) { return (in
 __device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p) {
     PfPlan plan;
     const int G = (int)gridDim.x;
-    plan.n_tp = pf_num_groups(p);
-    plan.n_items = plan.n_tp * p.Hkv;
+    plan.n_items = 0;
+    plan.longest = 0;
+    plan.shortest = 0x7fffffff;
+#pragma unroll
+    for (int j = 0; j < kMaxChunks; ++j) {
+        plan.items_before[j] = plan.n_items;
+        if (j < p.nchunks) {
+            const int n_tp = pf_num_groups(p.group, p.cC[j]);
+            plan.n_items += n_tp * p.Hkv;
+            if (n_tp > 0) {
+                plan.longest = max(plan.longest, pf_steps_of_rank(p.group, p.cP[j], p.cC[j], n_tp, 0));
+                plan.shortest = min(plan.shortest, pf_steps_of_rank(p.group, p.cP[j], p.cC[j], n_tp, n_tp - 1));
+            }
+        }
+    }
+    plan.items_before[kMaxChunks] = plan.n_items;
     const int r = plan.n_items % G;
     plan.n_whole = plan.n_items - r;
     plan.pieces = 1;
     if (r > 0) {
-        // the tail items are the shortest ones; size the pieces by the shortest of them
+        // the tail items are short ones; size the pieces by the shortest item
         // A piece costs its steps plus a merge that grows with k (about six steps' worth per piece merged), so
         // k ~ sqrt(steps / 6); never more pieces than fit side by side, never pieces shorter than the minimum.
-        const int shortest = pf_steps_of_rank(p, plan.n_tp, plan.n_tp - 1);
+        const int shortest = plan.shortest;
         int k = 1;
         while ((k + 1) * (k + 1) * 6 <= shortest) ++k;
         plan.pieces = max(1, min(min(G / r, k), shortest / kPfMinPieceSteps));
@@ -144,13 +162,22 @@ __device__ __forceinline__ PfItem pf_entry(const MixedParams& p, const PfPlan& p
         it.item = plan.n_whole + (entry - plan.n_whole) / plan.pieces;
         it.piece = (entry - plan.n_whole) % plan.pieces;
     }
-    const int rank = it.item / p.Hkv;
-    it.kvh = it.item % p.Hkv;
+    int chunk = 0;
+#pragma unroll
+    for (int j = 1; j < kMaxChunks; ++j)
+        if (j < p.nchunks && it.item >= plan.items_before[j]) chunk = j;
+    it.P = p.cP[chunk];
+    it.C = p.cC[chunk];
+    it.row0 = p.cRow0[chunk];
+    it.pages = p.prefill_pages + p.cPage0[chunk];
+    const int local = it.item - plan.items_before[chunk];
+    const int rank = local / p.Hkv;
+    it.kvh = local % p.Hkv;
     const int tt = 128 / p.group;
-    const int tp = plan.n_tp - 1 - rank;
+    const int tp = pf_num_groups(p.group, it.C) - 1 - rank;
     for (int t = 0; t < 2; ++t) {
         it.tok0[t] = (tp * 2 + t) * tt;
-        it.nkv[t] = pf_tiles_of(p, it.tok0[t]);
+        it.nkv[t] = pf_tiles_of(p.group, it.P, it.C, it.tok0[t]);
     }
     it.nk = max(it.nkv[0], it.nkv[1]);
     if (entry < plan.n_whole) {
@@ -181,18 +208,18 @@ __device__ __forceinline__ bool pf_produce(const CUtensorMap* kv_map, const CUte
             if (it.nkv[t] > it.j0)
                 for (int h = 0; h < G::kHalves; ++h)
                     tma_load_3d(sh.smem + G::kQOffset + t * G::kTileBytes + h * G::kHalfBytes, q_map, sh.bars + kBarQFull * 8,
-                                h * 64, it.kvh * p.group, it.tok0[t]);
+                                h * 64, it.kvh * p.group, it.row0 + it.tok0[t]);
     }
     // fused launch: tiles that reach into the chunk's own keys wait until every CTA has written its share of them
-    if (p.pool != nullptr && it.j1 * 128 > p.P && !wait_append(p)) {
+    if (p.pool != nullptr && it.j1 * 128 > it.P && !wait_append(p)) {
         if (lane == 0) {
             *sh.abort_flag = 1;
             report(p.ctrl, SW_ERR_DEVICE_TIMEOUT, kSiteWait, it.item);
         }
         return false;
     }
-    const int npages = (p.P + p.C + kPageSize - 1) / kPageSize;
-    auto page_of = [&](int j) { return (lane < 8 && j * 8 + lane < npages) ? p.prefill_pages[j * 8 + lane] : 0; };
+    const int npages = (it.P + it.C + kPageSize - 1) / kPageSize;
+    auto page_of = [&](int j) { return (lane < 8 && j * 8 + lane < npages) ? it.pages[j * 8 + lane] : 0; };
     int id_next = page_of(it.j0);
     for (int j = it.j0; j < it.j1; ++j, ++kv_it) {
         const uint32_t s = kv_it & 1, n = kv_it >> 1;
@@ -226,7 +253,7 @@ template <int D>
 __device__ __forceinline__ bool pf_sanitize(const MixedParams& p, const PfShared& sh, const PfItem& it, uint32_t& kv_it) {
     using G = PfGeo<D>;
     const int lane = threadIdx.x & 31;
-    const int kv_total = p.P + p.C;
+    const int kv_total = it.P + it.C;
     for (int j = it.j0; j < it.j1; ++j, ++kv_it) {
         const uint32_t s = kv_it & 1, n = kv_it >> 1;
         if (!pf_wait(sh, kBarVLanded + s, n & 1, p.ctrl, 3)) return false;
@@ -391,7 +418,7 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
     const int row = (warp & 3) * 32 + lane;
     const int tok = it.tok0[t] + row / p.group;
     const int head = it.kvh * p.group + row % p.group;
-    const int pos = p.P + tok;
+    const int pos = it.P + tok;
     const uint32_t lane_addr = sh.tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t s_addr = lane_addr + t * 128;  // P (bf16) aliases the first 64 columns of S
     const uint32_t o_addr = lane_addr + 256 + t * D;
@@ -498,8 +525,9 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
     if (!pf_wait(sh, kBarODone + t, (st.o_cnt + (j_end - it.j0) - 1) & 1, p.ctrl, 11)) return false;
     st.o_cnt += j_end - it.j0;
     tc_fence_after_sync();
-    const bool row_ok = tok < p.C;
-    __nv_bfloat16* dst = p.out + ((int64_t)tok * p.Hq + head) * D;
+    const bool row_ok = tok < it.C;
+    const int64_t out_row = (int64_t)it.row0 + tok;
+    __nv_bfloat16* dst = p.out + (out_row * p.Hq + head) * D;
     const bool whole = it.j0 == 0 && j_end == it.nkv[t];  // this piece holds every step of the tile
     if (whole) {
         // epilogue of an item this CTA did alone: O / l -> bf16 -> out
@@ -520,7 +548,7 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
                 }
             }
         }
-        if (row_ok && p.lse) p.lse[(int64_t)tok * p.Hq + head] = (m_ref + __log2f(l_sum)) * 0.6931471805599453f;
+        if (row_ok && p.lse) p.lse[out_row * p.Hq + head] = (m_ref + __log2f(l_sum)) * 0.6931471805599453f;
         tc_fence_before_sync();
         return true;
     }
@@ -603,7 +631,7 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
             }
         }
     }
-    if (row_ok && p.lse) p.lse[(int64_t)tok * p.Hq + head] = (m_all + __log2f(l_all)) * 0.6931471805599453f;
+    if (row_ok && p.lse) p.lse[out_row * p.Hq + head] = (m_all + __log2f(l_all)) * 0.6931471805599453f;
     return true;
 }
 

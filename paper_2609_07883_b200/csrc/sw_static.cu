@@ -91,7 +91,7 @@ extern "C" sw_status sw_decode_attn_static(const sw_layout* layout, int device, 
     if (!(g == 1 || g == 2 || g == 4 || g == 8)) return sw_fail(SW_ERR_UNSUPPORTED, "sw_decode_attn_static: unsupported head ratio");
     if (l.num_kv_heads > kStaticMaxKvHeads)
         return sw_fail(SW_ERR_WORKSPACE, "sw_decode_attn_static: at most %d KV heads fit the static scratch", kStaticMaxKvHeads);
-    if (batch->chunk_len != 0)
+    if (batch->chunk_len != 0 || batch->num_chunks != 0)
         return sw_fail(SW_ERR_UNSUPPORTED, "sw_decode_attn_static: decode-only (chunk_len must be 0)");
     if (batch->num_decode < 0 || batch->num_decode > kStaticMaxDecode)
         return sw_fail(SW_ERR_WORKSPACE, "sw_decode_attn_static: num_decode %d exceeds the static limit %d", batch->num_decode,
@@ -126,7 +126,6 @@ extern "C" sw_status sw_decode_attn_static(const sw_layout* layout, int device, 
     p.num_pages = l.num_pages;
     p.sm_scale = l.sm_scale > 0.f ? l.sm_scale : 1.0f / std::sqrt((float)l.head_dim);
     p.sm_scale_log2 = p.sm_scale * 1.4426950408889634f;
-    p.P = 0;
     p.C = 0;
     p.n = batch->num_decode;
     p.decode_kv_len = batch->decode_kv_len;

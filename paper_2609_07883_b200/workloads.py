@@ -92,6 +92,23 @@ class MixedBatch:
     decode_pages: np.ndarray  # int32 [indptr[n]]
     name: str = ""
     meta: dict = field(default_factory=dict)
+    # Several prefill chunks (of different prompts) in one iteration: chunk j has chunk_lens[j] tokens at prefix
+    # chunk_prefix_lens[j]; its rows follow chunk j-1's and its prompt's pages are
+    # prefill_pages[chunk_page_indptr[j]:chunk_page_indptr[j+1]].  chunk_len is then the sum of the chunk lengths and
+    # prefix_len the first chunk's.  None = the single chunk (prefix_len, chunk_len).
+    chunk_prefix_lens: np.ndarray | None = None
+    chunk_lens: np.ndarray | None = None
+    chunk_page_indptr: np.ndarray | None = None
+
+    def chunks(self):
+        """[(P, C, first row, page list)] of the iteration's prefill chunks (one entry for a single-chunk batch)."""
+        if self.chunk_lens is None:
+            return [(self.prefix_len, self.chunk_len, 0, self.prefill_pages)] if self.chunk_len > 0 else []
+        out, row = [], 0
+        for j, (P, C) in enumerate(zip(self.chunk_prefix_lens, self.chunk_lens)):
+            out.append((int(P), int(C), row, self.prefill_pages[self.chunk_page_indptr[j]:self.chunk_page_indptr[j + 1]]))
+            row += int(C)
+        return out
 
     @property
     def num_decode(self) -> int:
@@ -131,6 +148,26 @@ def make_batch(shape: AttnShape, num_pages: int, decode_lens, prefix_len: int, c
                       chunk_len=int(chunk_len), prefill_pages=ids[indptr[-1]:].copy(),
                       decode_kv_len=decode_lens.copy(), decode_page_indptr=indptr,
                       decode_pages=ids[:indptr[-1]].copy(), name=name)
+
+
+def make_multi_batch(shape: AttnShape, num_pages: int, decode_lens, chunks, rng: np.random.Generator,
+                     name: str = "") -> MixedBatch:
+    """As ``make_batch`` with several prefill chunks ``[(prefix_len, chunk_len), ...]``, each of its own prompt."""
+    chunks = [(int(P), int(C)) for P, C in chunks]
+    S = shape.page_size
+    base = make_batch(shape, num_pages, decode_lens, 0, 0, rng, name=name)
+    used = set(int(x) for x in base.decode_pages)
+    free = np.array([i for i in rng.permutation(num_pages) if int(i) not in used], dtype=np.int32)
+    per = [_cdiv(P + C, S) for P, C in chunks]
+    if sum(per) > len(free):
+        raise ValueError(f"batch needs {sum(per)} more pages, pool has {len(free)} free")
+    indptr = np.zeros(len(chunks) + 1, dtype=np.int32)
+    indptr[1:] = np.cumsum(per)
+    return MixedBatch(shape=shape, num_pages=int(num_pages), prefix_len=chunks[0][0], chunk_len=sum(C for _, C in chunks),
+                      prefill_pages=free[:indptr[-1]].copy(), decode_kv_len=base.decode_kv_len,
+                      decode_page_indptr=base.decode_page_indptr, decode_pages=base.decode_pages, name=name,
+                      chunk_prefix_lens=np.array([P for P, _ in chunks], dtype=np.int32),
+                      chunk_lens=np.array([C for _, C in chunks], dtype=np.int32), chunk_page_indptr=indptr)
 
 
 def normal_bf16_bits(rng: np.random.Generator, *size: int) -> np.ndarray:
