@@ -170,6 +170,51 @@ class Table:
         return int(chunk.value), int(flags.value), int(budget.value)
 
 
+def choose_first_fit(table: Table, now_ns, deadlines_ns, total_ctx, prefix_lens, remaining, c_max=4096, quantum=1,
+                     margin_abs_ns=0, margin_ppm=0, max_chunks=8):
+    """Several prefills in one iteration by first fit (Sec. 3.3, "Prefill batching"), written out by exhaustive scan.
+
+    Pending requests are taken oldest first.  With t tokens already admitted and the sum S of the admitted requests'
+    prefix lengths, request j may add c tokens if T^(n, ctx, S + prefix_j, t + c) + delta <= B (the prediction for the
+    total number of prefill tokens at the summed prefix bounds both the arithmetic and the K/V traffic of the separate
+    chunks from above).  The largest such c in {multiples of the quantum, <= L_j} with L_j = min(C_max - t,
+    remaining_j) is taken; a request that is admitted whole is followed by the next one, a request that is cut (or
+    gets nothing) ends the list.  Without active decodes there is no deadline: requests are admitted whole up to
+    C_max tokens.  Returns (chunks list, budget_ns)."""
+    dl = [int(x) for x in deadlines_ns]
+    n = len(dl)
+    budget = max(0, min(dl) - int(now_ns)) if n else 0
+    chunks, t, prefix_sum = [], 0, 0
+    q = max(1, int(quantum))
+
+    def cost(prefix, c):
+        raw = table.lookup(n, total_ctx, prefix, c)
+        if raw >= INF:
+            return INF
+        return raw + margin_abs_ns + -(-raw * margin_ppm // 1_000_000)
+
+    for j in range(min(len(remaining), max_chunks)):
+        L = min(c_max - t, int(remaining[j]))
+        if L <= 0:
+            break
+        if n == 0:
+            c = L - L % q
+        else:
+            c = 0
+            for cand in range(L - L % q, 0, -q):
+                if cost(prefix_sum + int(prefix_lens[j]), t + cand) <= budget:
+                    c = cand
+                    break
+        if c == 0:
+            break
+        chunks.append(c)
+        t += c
+        prefix_sum += int(prefix_lens[j])
+        if c < int(remaining[j]):
+            break
+    return chunks, budget
+
+
 def analytic_cost_ns(n: int, c: int) -> int:
     return int(lib().swo_analytic_cost_ns(int(n), int(c)))
 
