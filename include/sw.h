@@ -216,6 +216,21 @@ typedef struct {
     int32_t queries;      /* cost-model queries made by the bisection */
 } sw_choice;
 
+/* Several prefills in one iteration by first fit (Sec. 3.3, "Prefill batching").  The pending requests are given
+ * oldest first (HOST arrays prefix_lens / remaining_prefill, num_pending entries; at most SW_MAX_CHUNKS are looked at).
+ * With t tokens admitted so far and S the sum of the admitted requests' prefix lengths, request j may add c tokens if
+ * T^(n, ctx, S + prefix_lens[j], t + c) + delta <= B: the prediction for the total number of prefill tokens at the
+ * summed prefix bounds the arithmetic and the K/V traffic of the separate chunks from above.  A request that fits
+ * whole (L_j = min(C_max - t, remaining_j) tokens) is followed by the next; the first one that does not is cut by the
+ * bisection of Algorithm 1 and ends the list, so the search stays logarithmic.  Without active decodes requests are
+ * admitted whole up to C_max tokens.  chunks receives the admitted lengths (room for SW_MAX_CHUNKS), *num_chunks their
+ * count; out->chunk is their sum, out->predicted_ns the prediction for the admitted list.  With one pending request
+ * the result equals sw_choose_chunk's. */
+sw_status sw_choose_chunks(const sw_cost_table* table, const sw_chooser_params* params, int64_t now_ns,
+                           const int64_t* deadlines_ns, int32_t n_active, int64_t total_ctx, const int32_t* prefix_lens,
+                           const int32_t* remaining_prefill, int32_t num_pending, int32_t* chunks, int32_t* num_chunks,
+                           sw_choice* out);
+
 /* ---- telemetry (host only; no CUDA) --------------------------------------------------------------- */
 
 /* Residual table of the online feedback loop (Table 1 "Telemetry"; Sec. 3.3 "Prediction error"; Sec. 5.1).  Every

@@ -64,7 +64,7 @@ class sw_telemetry_totals(C.Structure):
 
 EXPORTS = ["sw_workspace_bytes", "sw_create", "sw_destroy", "sw_kv_append", "sw_mixed_attn_run", "sw_mixed_iteration_run",
            "sw_mixed_iteration_host", "sw_cost_probe", "sw_cost_probe_iteration", "sw_check_status", "sw_cost_table_create",
-           "sw_cost_table_destroy", "sw_cost_table_lookup", "sw_choose_chunk", "sw_last_error",
+           "sw_cost_table_destroy", "sw_cost_table_lookup", "sw_choose_chunk", "sw_choose_chunks", "sw_last_error",
            "sw_decode_attn_static", "sw_selftest_wait_timeout", "sw_telemetry_create", "sw_telemetry_destroy",
            "sw_telemetry_record", "sw_telemetry_margin", "sw_telemetry_exceeds", "sw_telemetry_get_totals"]
 
@@ -88,6 +88,8 @@ _lib.sw_check_status.argtypes = [_vp, _vp, C.POINTER(_i32), C.POINTER(_i32)]
 _lib.sw_cost_table_create.argtypes = [C.POINTER(_i32), _i32, C.POINTER(_i64), _i32, C.POINTER(_i32), _i32,
                                       C.POINTER(_i32), _i32, C.POINTER(_i64), C.c_int, C.c_int, C.POINTER(_vp)]
 _lib.sw_cost_table_destroy.argtypes = [_vp]
+_lib.sw_choose_chunks.argtypes = [_vp, C.POINTER(sw_chooser_params), _i64, C.POINTER(_i64), _i32, _i64, C.POINTER(_i32),
+                                  C.POINTER(_i32), _i32, C.POINTER(_i32), C.POINTER(_i32), C.POINTER(sw_choice)]
 _lib.sw_telemetry_create.argtypes = [C.POINTER(_i32), _i32, C.POINTER(_i32), _i32, _i32, C.POINTER(_vp)]
 _lib.sw_telemetry_destroy.argtypes = [_vp]
 _lib.sw_telemetry_destroy.restype = None
@@ -308,6 +310,28 @@ class CostTable:
 
     def __del__(self):
         self.close()
+
+
+SW_MAX_CHUNKS = 8
+
+
+def sw_choose_chunks(table, now_ns: int, deadlines_ns, total_ctx: int, prefix_lens, remaining_prefill, c_max: int = 4096,
+                     chunk_quantum: int = 1, margin_abs_ns: int = 0, margin_ppm: int = 0):
+    """First fit over the pending requests (oldest first).  Returns (list of admitted chunk lengths, sw_choice)."""
+    dl = np.ascontiguousarray(deadlines_ns, dtype=np.int64)
+    pre = np.ascontiguousarray(prefix_lens, dtype=np.int32)
+    rem = np.ascontiguousarray(remaining_prefill, dtype=np.int32)
+    if pre.shape != rem.shape:
+        raise ValueError("prefix_lens and remaining_prefill differ in length")
+    params = sw_chooser_params(margin_abs_ns, margin_ppm, c_max, chunk_quantum)
+    chunks = np.zeros(SW_MAX_CHUNKS, dtype=np.int32)
+    count = _i32(0)
+    out = sw_choice()
+    pi32 = lambda a: a.ctypes.data_as(C.POINTER(_i32))
+    _check(_lib.sw_choose_chunks(table.handle if table is not None else None, C.byref(params), now_ns,
+                                 dl.ctypes.data_as(C.POINTER(_i64)), len(dl), total_ctx, pi32(pre), pi32(rem), len(rem),
+                                 pi32(chunks), C.byref(count), C.byref(out)), "sw_choose_chunks")
+    return [int(x) for x in chunks[:count.value]], out
 
 
 class Telemetry:

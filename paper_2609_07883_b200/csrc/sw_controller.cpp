@@ -209,4 +209,84 @@ sw_status sw_choose_chunk(const sw_cost_table* table, const sw_chooser_params* p
     return SW_OK;
 }
 
+// Several prefills per iteration by first fit: requests oldest first, each admitted whole while the prediction for the
+// total still meets the budget; the first one that does not fit whole is cut by the bisection of Algorithm 1 and ends
+// the list.
+sw_status sw_choose_chunks(const sw_cost_table* table, const sw_chooser_params* params, int64_t now_ns,
+                           const int64_t* deadlines_ns, int32_t n_active, int64_t total_ctx, const int32_t* prefix_lens,
+                           const int32_t* remaining_prefill, int32_t num_pending, int32_t* chunks, int32_t* num_chunks,
+                           sw_choice* out) {
+    if (!params || !out || !chunks || !num_chunks || num_pending < 0 || (num_pending > 0 && (!prefix_lens || !remaining_prefill)))
+        return sw_fail(SW_ERR_INVALID_ARG, "sw_choose_chunks: null argument");
+    if (n_active < 0 || total_ctx < 0 || params->c_max < 0 || params->margin_ppm < 0 || params->margin_abs_ns < 0 ||
+        (n_active > 0 && !deadlines_ns))
+        return sw_fail(SW_ERR_INVALID_ARG, "sw_choose_chunks: negative size or missing deadlines");
+    for (int32_t j = 0; j < num_pending; ++j)
+        if (prefix_lens[j] < 0 || remaining_prefill[j] < 0)
+            return sw_fail(SW_ERR_INVALID_ARG, "sw_choose_chunks: negative length of pending request %d", j);
+    const int32_t q = params->chunk_quantum > 1 ? params->chunk_quantum : 1;
+    *out = sw_choice{0, 0, 0, 0, 0};
+    *num_chunks = 0;
+    if (num_pending == 0 || remaining_prefill[0] == 0) {
+        out->flags = SW_F_NO_PREFILL;
+        return SW_OK;
+    }
+    int64_t B = 0;
+    if (n_active > 0) {
+        if (!table) return sw_fail(SW_ERR_INVALID_ARG, "sw_choose_chunks: a cost table is required when decodes are active");
+        const int64_t earliest = *std::min_element(deadlines_ns, deadlines_ns + n_active);
+        B = earliest > now_ns ? earliest - now_ns : 0;
+        out->budget_ns = B;
+        int64_t t_raw = 0;
+        sw_status st = lookup(*table, n_active, total_ctx, 0, 0, &t_raw);
+        if (st != SW_OK) return st;
+        const int64_t decode_only = add_margin(t_raw, *params);
+        if (decode_only > B) out->flags |= SW_F_DECODE_INFEASIBLE;
+        out->predicted_ns = decode_only;
+    } else {
+        out->flags |= SW_F_NO_DECODE;
+    }
+    int64_t tokens = 0, prefix_sum = 0;
+    const int32_t limit = std::min<int32_t>(num_pending, SW_MAX_CHUNKS);
+    for (int32_t j = 0; j < limit; ++j) {
+        const int64_t room = (int64_t)params->c_max - tokens;
+        const int32_t L = (int32_t)std::min<int64_t>(room, remaining_prefill[j]);
+        if (L <= 0) break;
+        if ((int64_t)params->c_max - tokens < remaining_prefill[j]) out->flags |= SW_F_CAPPED;
+        int32_t c = 0;
+        if (n_active == 0) {
+            c = L - L % q;
+        } else {
+            const int64_t prefix = prefix_sum + prefix_lens[j];
+            // upper-mid bisection over k in [0, L/q], c = k*q (Algorithm 1 with the tokens admitted so far as offset)
+            int32_t lo = 0, hi = L / q;
+            int64_t predicted_at_lo = out->predicted_ns;
+            while (lo < hi) {
+                const int32_t mid = lo + (hi - lo + 1) / 2;
+                int64_t t_raw = 0;
+                sw_status st = lookup(*table, n_active, total_ctx, prefix, tokens + (int64_t)mid * q, &t_raw);
+                if (st != SW_OK) return st;
+                out->queries += 1;
+                const int64_t t = add_margin(t_raw, *params);
+                if (t <= B) {
+                    lo = mid;
+                    predicted_at_lo = t;
+                } else {
+                    hi = mid - 1;
+                }
+            }
+            c = lo * q;
+            if (c > 0) out->predicted_ns = predicted_at_lo;
+        }
+        if (c == 0) break;
+        chunks[*num_chunks] = c;
+        *num_chunks += 1;
+        tokens += c;
+        prefix_sum += prefix_lens[j];
+        if (c < remaining_prefill[j]) break;
+    }
+    out->chunk = (int32_t)tokens;
+    return SW_OK;
+}
+
 }  // extern "C"

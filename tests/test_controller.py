@@ -134,3 +134,38 @@ def test_raw_non_monotone_table_breaks_bisection_and_cummax_restores_it(B, oracl
     lt = B.CostTable([1], [10], [0], grid, raw, make_monotone=True)
     for budget, _want_raw, want_mono in rows[3:]:
         assert B.sw_choose_chunk(lt, 0, [budget], 10, 0, 112, c_max=112).chunk == want_mono
+
+
+def test_first_fit_over_several_pending_requests_matches_the_oracle(B, oracle):
+    """sw_choose_chunks against the oracle's exhaustive scan on random monotone tables (bit-exact lists and budget)."""
+    rng = np.random.default_rng(21)
+    for trial in range(12):
+        grids = random_table(rng, monotone_input=False)
+        lt, ot = both_tables(B, oracle, *grids)
+        n_grid, ctx_grid, prefix_grid, chunk_grid, _ = grids
+        values = sorted(set(int(v) for v in ot.cost.reshape(-1)))
+        for _ in range(40):
+            n = int(rng.integers(0, n_grid[-1] + 1))
+            ctx = int(rng.integers(0, ctx_grid[-1] + 1))
+            m = int(rng.integers(1, 11))
+            # keep the summed prefixes inside the table's prefix axis
+            prefixes = [int(x) for x in rng.integers(0, max(1, int(prefix_grid[-1]) // 10) + 1, size=m)]
+            remaining = [int(x) for x in rng.integers(1, int(chunk_grid[-1]) + 50, size=m)]
+            c_max = int(rng.integers(1, int(chunk_grid[-1]) + 100))
+            quantum = int(rng.choice([1, 1, 16]))
+            now = int(rng.integers(0, 10**6))
+            budget = int(rng.choice(values)) + int(rng.integers(-2, 3)) if rng.integers(0, 4) else int(rng.integers(0, 10**12))
+            dl = now + max(0, budget) + rng.integers(0, 5 * MS, size=n)
+            if n:
+                dl[rng.integers(0, n)] = now + max(0, budget)
+            mabs, mppm = int(rng.integers(0, 1000)), int(rng.choice([0, 50_000]))
+            got, ch = B.sw_choose_chunks(lt if n else None, now, dl, ctx, prefixes, remaining, c_max=c_max,
+                                         chunk_quantum=quantum, margin_abs_ns=mabs, margin_ppm=mppm)
+            want, want_budget = oracle.choose_first_fit(ot, now, dl, ctx, prefixes, remaining, c_max=c_max, quantum=quantum,
+                                                        margin_abs_ns=mabs, margin_ppm=mppm)
+            assert got == want, (trial, n, prefixes, remaining, c_max, quantum, budget)
+            assert ch.chunk == sum(want) and ch.budget_ns == want_budget
+            if m == 1 and n > 0:
+                one = B.sw_choose_chunk(lt, now, dl, ctx, prefixes[0], remaining[0], c_max=c_max, chunk_quantum=quantum,
+                                        margin_abs_ns=mabs, margin_ppm=mppm)
+                assert ([one.chunk] if one.chunk else []) == got and one.predicted_ns == ch.predicted_ns
