@@ -88,7 +88,8 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
               c_max: int = 4096, margin_ppm: int = 50_000, margin_abs_ns: int = 0, quantum: int = 16, max_decode: int = 512,
               ctx_cap: int | None = None, seed: int = W.SEED_BASE + 44, log=None, page_tables: bool = True,
               ttft_slo_ms: float | None = None, telemetry=None, fallback_margin_ns: int | None = None,
-              residual_percentile_ppm: int = 990_000, residual_min_samples: int = 8, fallback_hold: int = 8) -> dict:
+              residual_percentile_ppm: int = 990_000, residual_min_samples: int = 8, fallback_hold: int = 8,
+              max_prefills: int = 1, prefix_cap: int | None = None) -> dict:
     """Run the whole trace; returns statistics.  ``policy`` is "sloweave" or "fixed:<chunk>".  ``execute(batch)`` runs
     one iteration and returns its duration in ns (``gpu_executor`` for the CUDA path).  ``ctx_cap`` clamps the total
     context passed to the table lookup to the table's last grid point.  ``page_tables=False`` hands ``execute`` a batch
@@ -99,7 +100,13 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
     prediction and measured duration are recorded, the residual table's margin for (n, L) is added to the controller's
     margin, and, when ``fallback_margin_ns`` is given and the residuals exceed it, the iteration runs decode-only.  So
     that a stale residual cannot starve the queue, at most ``fallback_hold`` consecutive iterations fall back; the next
-    one admits a chunk again under the residual margin and so refreshes the residuals."""
+    one admits a chunk again under the residual margin and so refreshes the residuals.
+
+    ``max_prefills > 1`` (SLOWeave policy only) admits several pending prompts per iteration by first fit
+    (``sw_choose_chunks``, Sec. 3.3 "Prefill batching"): whole prompts oldest first while the prediction for the total
+    still meets the budget, the first one that does not fit cut by the bisection; the iteration then carries one
+    prefill chunk per admitted prompt.  ``prefix_cap`` (the table's last prefix grid point) bounds the summed prefix
+    lengths of the candidates, which is the prefix coordinate the first-fit prediction is looked up at."""
     from . import binding as B
 
     S = shape.page_size
@@ -116,6 +123,7 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
     misses_chunk = misses_decode_only = infeasible_flags = stalled_for_memory = 0
     chunks, iter_ns, pred_err = [], [], []
     fallback_iters = fallback_run = 0
+    prompts_per_chunk_iter = []
     prefill_tokens = 0
     wall0 = time.time()
     while done < len(reqs):
@@ -144,6 +152,7 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
         budget = int(deadlines.min() - now) if n else 0
         predicted = 0
         flags = 0
+        admitted = None      # [(request, tokens)] when several prompts share the iteration
         fell_back = False
         extra_margin = 0
         if telemetry is not None and fixed_chunk is None and n and remaining:
@@ -158,6 +167,24 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
             fallback_iters += 1
         elif fixed_chunk is not None:
             c = min(fixed_chunk, remaining)
+        elif max_prefills > 1 and head is not None:
+            # first fit over the oldest pending requests (each needs its blocks reserved before it can be scheduled)
+            cands, prefix_total = [], 0
+            for r in list(pending)[:min(max_prefills, B.SW_MAX_CHUNKS, max(1, max_decode - n))]:
+                if cands and prefix_cap is not None and prefix_total + r.prefilled > prefix_cap:
+                    break
+                prefix_total += r.prefilled
+                if r.pages is None:
+                    r.pages = pool.take(-(-(r.prompt + r.output) // S))
+                    if r.pages is None:
+                        break
+                cands.append(r)
+            fallback_run = 0
+            lens_adm, ch = B.sw_choose_chunks(table if n else None, now, deadlines, total_ctx, [r.prefilled for r in cands],
+                                              [r.prompt - r.prefilled for r in cands], c_max=c_max, chunk_quantum=1,
+                                              margin_abs_ns=margin_abs_ns + extra_margin, margin_ppm=margin_ppm)
+            admitted = list(zip(cands, lens_adm))
+            c, flags, predicted = ch.chunk, ch.flags, ch.predicted_ns
         else:
             q_eff = quantum if remaining >= quantum else 1   # the last few tokens of a prompt are below the quantum
             prefilled = head.prefilled if head else 0
@@ -181,7 +208,9 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
                 continue
             raise RuntimeError("serving loop stalled: pool too small for the remaining requests")
         # ---- build the iteration and run it over the layer stack -----------------------------------------------
-        P = head.prefilled if (head is not None and c > 0) else 0
+        if admitted is None:
+            admitted = [(head, c)] if c > 0 else []
+        P = admitted[0][0].prefilled if admitted else 0
         lens = np.array([r.prompt + r.generated for r in active], dtype=np.int32)
         per = [(-(-int(L) // S)) for L in lens]
         indptr = np.zeros(n + 1, dtype=np.int32)
@@ -192,7 +221,18 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
             ppages = np.asarray(head.pages[: -(-(P + c) // S)], dtype=np.int32) if c > 0 else np.zeros(0, np.int32)
         else:
             dpages = ppages = np.zeros(0, np.int32)
-        batch = W.MixedBatch(shape, num_pages, P, c, ppages, lens, indptr, dpages)
+        if len(admitted) > 1:
+            # one chunk per admitted prompt, the longest (prefix + chunk) first: that is the order they are scheduled in
+            order = sorted(admitted, key=lambda rc: -(rc[0].prefilled + rc[1]))
+            lists = [np.asarray(r.pages[: -(-(r.prefilled + cj) // S)], dtype=np.int32) if page_tables else
+                     np.zeros(0, np.int32) for r, cj in order]
+            cp_indptr = np.zeros(len(order) + 1, dtype=np.int32)
+            cp_indptr[1:] = np.cumsum([len(x) for x in lists])
+            batch = W.MixedBatch(shape, num_pages, order[0][0].prefilled, c, np.concatenate(lists), lens, indptr, dpages,
+                                 chunk_prefix_lens=np.array([r.prefilled for r, _ in order], dtype=np.int32),
+                                 chunk_lens=np.array([cj for _, cj in order], dtype=np.int32), chunk_page_indptr=cp_indptr)
+        else:
+            batch = W.MixedBatch(shape, num_pages, P, c, ppages, lens, indptr, dpages)
         dt = int(execute(batch))
         now += dt
         iters += 1
@@ -208,7 +248,8 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
         if predicted and n:
             pred_err.append(dt - predicted)
         if telemetry is not None and n:
-            raw = table.lookup(n, total_ctx, P, c)      # the table's own prediction, without any margin
+            # the table's own prediction, without any margin (several chunks: total tokens at the summed prefix)
+            raw = table.lookup(n, total_ctx, sum(r.prefilled for r, _ in admitted) if admitted else 0, c)
             telemetry.record(n, c, raw, dt, slack_ns=budget - dt, fallback=fell_back)
         still = []
         for r in active:
@@ -227,8 +268,11 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
             chunk_iters += 1
             chunks.append(c)
             prefill_tokens += c
-            head.prefilled += c
+            prompts_per_chunk_iter.append(len(admitted))
+        for head, cj in admitted:                  # admitted prompts are the oldest pending ones, in queue order
+            head.prefilled += cj
             if head.prefilled >= head.prompt:      # the iteration that finishes the prompt emits the first token
+                assert pending[0] is head
                 pending.popleft()
                 head.first_token = now
                 head.last_token = now
@@ -265,6 +309,7 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
         "requests_meeting_tpot": int(np.sum(p99_gap <= tpot_ms)),
         "prediction_error_ms_p99": float(np.percentile(pred_err, 99)) / MS if pred_err else 0.0,
         "fallback_iterations": fallback_iters,
+        "mean_prompts_per_chunk_iteration": float(np.mean(prompts_per_chunk_iter)) if prompts_per_chunk_iter else 0.0,
         "margin_ppm": margin_ppm, "c_max": c_max, "quantum": quantum, "wall_s": time.time() - wall0,
     }
 
@@ -287,6 +332,7 @@ def main(argv=None):
     ap.add_argument("--margin-ppm", type=int, default=50_000)
     ap.add_argument("--table", default=None, help="JSON cost table to reuse; measured first when absent")
     ap.add_argument("--table-reps", type=int, default=8)
+    ap.add_argument("--max-prefills", type=int, default=1, help="prompts admitted per iteration (first fit when > 1)")
     ap.add_argument("--out", default="bursty_results.json")
     args = ap.parse_args(argv)
 
@@ -327,7 +373,8 @@ def main(argv=None):
             for policy in args.policies:
                 log(f"run: rate x{scale} tpot={tpot} ms policy={policy}")
                 res = run_trace(scaled, tpot, table, execute, shape, args.pages, policy=policy, c_max=args.c_max,
-                                margin_ppm=args.margin_ppm, max_decode=max_decode, ctx_cap=tab["ctx_grid"][-1], log=log)
+                                margin_ppm=args.margin_ppm, max_decode=max_decode, ctx_cap=tab["ctx_grid"][-1], log=log,
+                                max_prefills=args.max_prefills, prefix_cap=tab["prefix_grid"][-1])
                 B.sw_check_status(ctx)
                 res["rate_scale"] = scale
                 log(json.dumps(res))

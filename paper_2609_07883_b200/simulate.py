@@ -51,7 +51,11 @@ def analytic_table(max_decode: int, c_max: int, quantum: int):
 
 
 POLICIES = {"full": f"fixed:{FULL}", "fixed-64": "fixed:64", "fixed-256": "fixed:256", "fixed-1024": "fixed:1024",
-            "sloweave": "sloweave"}
+            "sloweave": "sloweave", "sloweave-8": "sloweave"}
+# "sloweave-8" admits up to eight pending prompts per iteration by first fit (Sec. 3.3, "Prefill batching"); the
+# paper's own study admits one, so it is not part of the default policy list.
+MAX_PREFILLS = {"sloweave-8": 8}
+DEFAULT_POLICIES = ["full", "fixed-64", "fixed-256", "fixed-1024", "sloweave"]
 
 
 def run_one(workload: str, policy: str, tpot_ms: float, seed: int, table, num_requests: int, c_max: int, quantum: int,
@@ -61,7 +65,8 @@ def run_one(workload: str, policy: str, tpot_ms: float, seed: int, table, num_re
     trace = W.study_trace(workload, seed, num_requests)
     res = serving.run_trace(trace, tpot_ms, table, lambda b: analytic_cost_ns(b.num_decode, b.chunk_len), W.LLAMA,
                             1 << 21, policy=POLICIES[policy], c_max=c_max, margin_ppm=0, quantum=quantum,
-                            max_decode=max_decode, page_tables=False, ttft_slo_ms=W.STUDY[workload]["ttft_slo_ms"])
+                            max_decode=max_decode, page_tables=False, ttft_slo_ms=W.STUDY[workload]["ttft_slo_ms"],
+                            max_prefills=MAX_PREFILLS.get(policy, 1))
     res["workload"], res["policy"], res["seed"] = workload, policy, seed
     return res
 
@@ -95,7 +100,7 @@ def ratios(means) -> list:
     for wl in sorted({m["workload"] for m in means}):
         for tpot in sorted({m["tpot_ms"] for m in means}):
             cell = {m["policy"]: m["goodput_rps"] for m in means if m["workload"] == wl and m["tpot_ms"] == tpot}
-            static = {k: v for k, v in cell.items() if k != "sloweave"}
+            static = {k: v for k, v in cell.items() if not k.startswith("sloweave")}
             if "sloweave" not in cell or not static:
                 continue
             best = max(static, key=static.get)
@@ -110,7 +115,7 @@ def main(argv=None):
 
     ap = argparse.ArgumentParser(description="simulator study: policies under the analytic cost model (CPU only)")
     ap.add_argument("--workloads", nargs="+", default=["chat", "mixed", "long", "bursty"], choices=sorted(W.STUDY))
-    ap.add_argument("--policies", nargs="+", default=list(POLICIES), choices=list(POLICIES))
+    ap.add_argument("--policies", nargs="+", default=DEFAULT_POLICIES, choices=list(POLICIES))
     ap.add_argument("--tpot-ms", type=float, nargs="+", default=[10.0, 25.0, 50.0])
     ap.add_argument("--seeds", type=int, default=5)
     ap.add_argument("--requests", type=int, default=1000)

@@ -81,3 +81,30 @@ def test_measured_table_is_made_monotone_and_drives_the_loop(setup):
     assert res["p99_chunk"] <= 512 and res["requests"] == 24
     assert res["deadline_misses_with_chunk"] == 0
     assert B.sw_check_status(ctx, raise_on_error=False) == (0, 0)
+
+
+def test_loop_with_several_prompts_per_iteration_on_the_device(setup):
+    """The serving loop with first fit over pending prompts, through the real executor: iterations with several prefill
+    chunks run on the device without a reported problem and every prompt token is prefilled exactly once."""
+    B, ctx, pools, shape, pages = setup
+    from paper_2609_07883_b200 import profiler, serving
+
+    n_grid, ctx_grid, prefix_grid, chunk_grid = [1, 8, 64], [2048, 30000], [0, 4096], [0, 64, 256, 512]
+    tab = profiler.measure_table(ctx, pools, shape, pages, n_grid, ctx_grid, prefix_grid, chunk_grid, reps=3, warmup=1,
+                                 fused=True)
+    table = profiler.to_cost_table(tab)
+    trace = W.bursty_trace(num_requests=40, rate_low=400.0, rate_high=2000.0, mean_dwell_s=0.05, prompt_median=150.0,
+                           prompt_clip=(8, 600), mean_output=10.0, rng=np.random.default_rng(8))
+    inner = serving.gpu_executor(ctx, pools, shape, 512, 64)
+    seen = []
+
+    def execute(batch):
+        seen.append(0 if batch.chunk_lens is None else len(batch.chunk_lens))
+        return inner(batch)
+
+    res = serving.run_trace(trace, 25.0, table, execute, shape, pages, policy="sloweave", c_max=512, max_decode=64,
+                            ctx_cap=ctx_grid[-1], max_prefills=8, prefix_cap=prefix_grid[-1])
+    assert res["prefill_tokens"] == int(trace["prompt_len"].sum())
+    assert max(seen) >= 2, "no iteration carried more than one prompt"
+    assert res["deadline_misses_with_chunk"] == 0
+    assert B.sw_check_status(ctx, raise_on_error=False) == (0, 0)

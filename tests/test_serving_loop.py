@@ -67,3 +67,32 @@ def test_arrivals_become_eligible_at_iteration_end_and_tokens_add_up(env):
     assert sum(n for n, _, _ in seen) == int(trace["output_len"].sum()) - int((trace["output_len"] >= 1).sum())
     assert sum(c for _, c, _ in seen) == int(trace["prompt_len"].sum())
     assert res["ttft_ms_p50"] > 0 and res["trace_duration_s"] * 1e9 >= trace["arrival_ns"][-1]
+
+
+def test_several_prompts_per_iteration_by_first_fit(env):
+    """max_prefills > 1: whole prompts are admitted oldest first while the total fits, the first that does not is cut;
+    every token is prefilled exactly once, no admitted list misses a deadline, and fewer iterations carry a chunk."""
+    B, serving, table, execute, trace = env
+    seen = []
+
+    def spy(batch):
+        seen.append(batch)
+        return execute(batch)
+
+    one = serving.run_trace(trace, 25.0, table, execute, W.LLAMA, 8192, policy="sloweave", c_max=2048, margin_ppm=0,
+                            quantum=16, max_decode=96)
+    many = serving.run_trace(trace, 25.0, table, spy, W.LLAMA, 8192, policy="sloweave", c_max=2048, margin_ppm=0,
+                             quantum=16, max_decode=96, max_prefills=8)
+    assert many["prefill_tokens"] == one["prefill_tokens"] == int(trace["prompt_len"].sum())
+    assert many["deadline_misses_with_chunk"] == 0
+    assert many["mean_prompts_per_chunk_iteration"] > 1.05
+    assert many["chunk_iterations"] < one["chunk_iterations"]
+    multi = [b for b in seen if b.chunk_lens is not None]
+    assert multi, "no iteration carried more than one prompt"
+    for b in multi:
+        assert 2 <= len(b.chunk_lens) <= 8 and int(b.chunk_lens.sum()) == b.chunk_len <= 2048
+        assert b.chunk_page_indptr[-1] == len(b.prefill_pages)
+        order = b.chunk_prefix_lens + b.chunk_lens
+        assert (np.diff(order) <= 0).all()               # the longest (prefix + chunk) first
+        for P, C, row0, pages in b.chunks():
+            assert len(pages) == -(-(P + C) // 16)
