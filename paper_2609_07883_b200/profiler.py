@@ -189,6 +189,46 @@ def sweep(config: str, reps: int, log) -> list:
     return rows
 
 
+def sweep_multichunk(reps: int, log) -> list:
+    """One iteration's prefill tokens given as 1, 2, 4 or 8 chunks of different prompts (each at its own prefix), with
+    and without the chat workload's 64 decodes: launch times of ``sw_mixed_attn_run``."""
+    import torch
+
+    from . import binding as B
+
+    dev = torch.device("cuda", 0)
+    shape = W.LLAMA
+    rows = []
+    for total, prefix in ((512, 512), (2048, 4096)):
+        for n in (0, 64):
+            for k in (1, 2, 4, 8):
+                rng = W.rng_for(1)
+                lens = rng.integers(256, 2048, size=n, endpoint=True) if n else []
+                chunks = [(prefix, total // k)] * k
+                need = sum(-(-int(x) // 16) for x in lens) + k * (-(-(prefix + total // k) // 16)) + 64
+                batch = W.make_multi_batch(shape, need, lens, chunks, rng)
+                pools = []
+                for layer in range(4):
+                    t = torch.empty(batch.num_pages * shape.page_elems, dtype=torch.bfloat16, device=dev)
+                    W.fill_normal_bf16_(t, W.SEED_BASE + 700 + layer)
+                    pools.append(t)
+                pages = int(batch.prefill_pages.shape[0] + batch.decode_pages.shape[0])
+                ctx = B.Context(shape, batch.num_pages, batch.chunk_len, max(n, 1), pages + 16)
+                q = torch.randn(batch.num_rows, shape.num_q_heads, shape.head_dim, device=dev).to(torch.bfloat16)
+                out = torch.empty_like(q)
+                p50, p99, _ = B.sw_cost_probe(ctx, pools, B.DeviceBatch(batch, dev), q, out, warmup=2, reps=reps)
+                B.sw_check_status(ctx)
+                flops = 4 * shape.num_q_heads * shape.head_dim * k * ((total // k) * prefix + (total // k) * (total // k + 1) // 2)
+                row = {"prefill_tokens": total, "prefix_of_each": prefix, "chunks": k, "decodes": n, "us_p50": p50 / 4e3,
+                       "us_p99": p99 / 4e3, "prefill_gflop": flops / 1e9}
+                rows.append(row)
+                log(f"tokens {total:5d} in {k} chunk(s) at prefix {prefix:5d}, {n:3d} decodes: {row['us_p50']:8.1f} us "
+                    f"(p99 {row['us_p99']:.1f}), {flops / 1e9:.1f} GFLOP of prefill")
+                del ctx, pools
+                torch.cuda.empty_cache()
+    return rows
+
+
 def main(argv=None):
     import argparse
     import sys
@@ -196,12 +236,15 @@ def main(argv=None):
     from . import build
 
     ap = argparse.ArgumentParser(description="cost surface of a named workload: mixed / prefill-only / decode-only launches")
-    ap.add_argument("--config", choices=["chat", "mixed", "long"], default="mixed")
+    ap.add_argument("--config", choices=["chat", "mixed", "long", "multichunk"], default="mixed")
     ap.add_argument("--reps", type=int, default=10)
     ap.add_argument("--out", default=None)
     args = ap.parse_args(argv)
     build.build()
-    rows = sweep(args.config, args.reps, lambda s: print(s, flush=True))
+    if args.config == "multichunk":
+        rows = sweep_multichunk(args.reps, lambda s: print(s, flush=True))
+    else:
+        rows = sweep(args.config, args.reps, lambda s: print(s, flush=True))
     out = args.out or f"cost_surface_{args.config}.json"
     Path(out).parent.mkdir(parents=True, exist_ok=True)
     Path(out).write_text(json.dumps(rows, indent=1))
