@@ -41,10 +41,12 @@ class PagePool:
 
 class Request:
     __slots__ = ("rid", "arrival", "prompt", "output", "prefilled", "generated", "pages", "last_token", "first_token",
-                 "gaps", "done_at")
+                 "gaps", "done_at", "D_ns", "margin_ns")
 
-    def __init__(self, rid, arrival, prompt, output):
+    def __init__(self, rid, arrival, prompt, output, D_ns, margin_ns=0):
         self.rid, self.arrival, self.prompt, self.output = rid, int(arrival), int(prompt), int(output)
+        self.D_ns = int(D_ns)            # the request's own token-gap objective D_i (Sec. 3.4, heterogeneous SLOs)
+        self.margin_ns = int(margin_ns)  # the prediction margin delta_i reserved for its class
         self.prefilled = 0
         self.generated = 0
         self.pages = None
@@ -113,7 +115,12 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
     D_ns = int(tpot_ms * MS)
     rng = np.random.default_rng(seed)
     pool = PagePool(num_pages, rng)
-    reqs = [Request(i, trace["arrival_ns"][i], trace["prompt_len"][i], trace["output_len"][i])
+    # per-request objectives D_i and class margins delta_i (optional trace columns "tpot_ms" / "margin_ms")
+    tpot_of = trace.get("tpot_ms")
+    margin_of = trace.get("margin_ms")
+    reqs = [Request(i, trace["arrival_ns"][i], trace["prompt_len"][i], trace["output_len"][i],
+                    (float(tpot_of[i]) if tpot_of is not None else tpot_ms) * MS,
+                    (float(margin_of[i]) if margin_of is not None else 0.0) * MS)
             for i in range(len(trace["arrival_ns"]))]
     fixed_chunk = int(policy.split(":")[1]) if policy.startswith("fixed:") else None
 
@@ -145,7 +152,9 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
         if n >= max_decode and head is not None:
             head = None                             # the decode batch is full: no new request can finish its prefill
         remaining = head.prompt - head.prefilled if head is not None else 0
-        deadlines = np.array([r.last_token + D_ns for r in active], dtype=np.int64)
+        # d_i = l_i + D_i, less the margin delta_i reserved for the request's class: B = min_i(d_i - delta_i) - now
+        deadlines = np.array([r.last_token + r.D_ns - r.margin_ns for r in active], dtype=np.int64)
+        true_deadline = min((r.last_token + r.D_ns for r in active), default=0)
         total_ctx = sum(r.prompt + r.generated for r in active)
         if ctx_cap is not None:
             total_ctx = min(total_ctx, ctx_cap)
@@ -238,7 +247,7 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
         iters += 1
         iter_ns.append(dt)
         # ---- bookkeeping ------------------------------------------------------------------------------------------
-        if n and dt > budget:
+        if n and now > true_deadline:
             if c > 0:
                 misses_chunk += 1
             else:
@@ -290,9 +299,10 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
     ttft = np.array([r.first_token - r.arrival for r in reqs], dtype=np.float64) / MS
     p99_gap = np.array([np.percentile(r.gaps, 99) if r.gaps else 0.0 for r in reqs]) / MS
     duration_s = now / 1e9
+    tpot_each = np.array([r.D_ns for r in reqs], dtype=np.float64) / MS
     slo = {}
     if ttft_slo_ms is not None:
-        both = int(np.sum((ttft <= ttft_slo_ms) & (p99_gap <= tpot_ms)))
+        both = int(np.sum((ttft <= ttft_slo_ms) & (p99_gap <= tpot_each)))
         slo = {"ttft_slo_ms": ttft_slo_ms, "requests_meeting_both_slos": both, "slo_attainment": both / len(reqs),
                "goodput_rps": both / duration_s, "throughput_rps": len(reqs) / duration_s}
     return {
@@ -306,7 +316,7 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
         "iter_ms_p50": float(np.percentile(iter_ns, 50)) / MS, "iter_ms_p99": float(np.percentile(iter_ns, 99)) / MS,
         "ttft_ms_p50": float(np.percentile(ttft, 50)), "ttft_ms_p99": float(np.percentile(ttft, 99)),
         "tpot_ms_p99_of_request_p99": float(np.percentile(p99_gap, 99)),
-        "requests_meeting_tpot": int(np.sum(p99_gap <= tpot_ms)),
+        "requests_meeting_tpot": int(np.sum(p99_gap <= tpot_each)),
         "prediction_error_ms_p99": float(np.percentile(pred_err, 99)) / MS if pred_err else 0.0,
         "fallback_iterations": fallback_iters,
         "mean_prompts_per_chunk_iteration": float(np.mean(prompts_per_chunk_iter)) if prompts_per_chunk_iter else 0.0,

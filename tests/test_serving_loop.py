@@ -96,3 +96,30 @@ def test_several_prompts_per_iteration_by_first_fit(env):
         assert (np.diff(order) <= 0).all()               # the longest (prefix + chunk) first
         for P, C, row0, pages in b.chunks():
             assert len(pages) == -(-(P + C) // 16)
+
+
+def test_heterogeneous_objectives_and_class_margins(env):
+    """Per-request objectives D_i (Sec. 3.4): a 10 ms interactive class shares the batch with a 50 ms class.  The budget
+    is the minimum over the active requests, so the tight class is protected whenever one of its requests is active and
+    the loose one never misses either; a class margin delta_i only tightens the budget."""
+    B, serving, table, execute, trace = env
+    rng = np.random.default_rng(12)
+    tight = rng.random(len(trace["arrival_ns"])) < 0.3
+    mixed = dict(trace, tpot_ms=np.where(tight, 10.0, 50.0))
+    res = serving.run_trace(mixed, 25.0, table, execute, W.LLAMA, 8192, policy="sloweave", c_max=2048, margin_ppm=0,
+                            quantum=16, max_decode=96)
+    assert res["deadline_misses_with_chunk"] == 0
+    assert res["requests_meeting_tpot"] == len(tight)            # every request meets its OWN objective
+    loose_only = serving.run_trace(dict(trace, tpot_ms=np.full(len(tight), 50.0)), 25.0, table, execute, W.LLAMA, 8192,
+                                   policy="sloweave", c_max=2048, margin_ppm=0, quantum=16, max_decode=96)
+    tight_only = serving.run_trace(dict(trace, tpot_ms=np.full(len(tight), 10.0)), 25.0, table, execute, W.LLAMA, 8192,
+                                   policy="sloweave", c_max=2048, margin_ppm=0, quantum=16, max_decode=96)
+    # the mixture sits between the two pure cases: slack of the loose class is used when no tight request is active
+    assert tight_only["mean_chunk"] <= res["mean_chunk"] <= loose_only["mean_chunk"]
+    assert tight_only["mean_chunk"] < loose_only["mean_chunk"]
+    # a 2 ms margin for the tight class shrinks the chunks further and still meets everything
+    guarded = serving.run_trace(dict(mixed, margin_ms=np.where(tight, 2.0, 0.0)), 25.0, table, execute, W.LLAMA, 8192,
+                                policy="sloweave", c_max=2048, margin_ppm=0, quantum=16, max_decode=96)
+    assert guarded["deadline_misses_with_chunk"] == 0 and guarded["requests_meeting_tpot"] == len(tight)
+    assert guarded["mean_chunk"] <= res["mean_chunk"]
+    assert guarded["tpot_ms_p99_of_request_p99"] <= 50.0
