@@ -1,10 +1,13 @@
 // sm_100a kernels of the mixed prefill-chunk + decode attention iteration.
 //
 //   sw_kv_append_kernel     scatter of this iteration's new K/V rows into their pages (Table 1, KV manager)
-//   sw_mixed_attn_kernel    ONE persistent launch per iteration (Sec. 4.1): every CTA plans the split-KV units
-//                           from the context lengths, warps pull units from a shared counter, stream K/V pages
-//                           with TMA into a per-warp shared-memory ring, keep an online softmax in registers and
-//                           the last-arriving warp of a request merges its partial results.
+//   sw_mixed_attn_kernel    ONE persistent launch per iteration (Sec. 4.1).  Optionally it first writes the new K/V
+//                           rows itself (the fused form of the append).  CTAs with chunk-prefill entries run them on
+//                           the tensor cores (sw_prefill.cuh).  Every CTA then plans the split-KV decode units from
+//                           the context lengths; a warp's first unit is fixed by its index, further ones come from a
+//                           shared counter; a unit streams its K/V pages with TMA into the warp's shared-memory ring
+//                           and keeps an online softmax in registers; of the units of one (request, kv head) the one
+//                           that drew the last ticket merges the partial results.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
