@@ -262,6 +262,9 @@ sw_status sw_telemetry_margin(const sw_telemetry* t, int32_t n, int32_t c, int32
  * scheduler then runs the iteration decode-only. */
 sw_status sw_telemetry_exceeds(const sw_telemetry* t, int32_t n, int32_t c, int32_t percentile_ppm, int32_t min_samples,
                                int64_t configured_margin_ns, int32_t* exceeds);
+/* Forgets every residual (the totals stay): to be called when the cost table the predictions come from is replaced
+ * (re-profiling, Sec. 5.1), since residuals against the old table say nothing about the new one. */
+sw_status sw_telemetry_reset(sw_telemetry* t);
 sw_status sw_telemetry_get_totals(const sw_telemetry* t, sw_telemetry_totals* out);
 
 /* Algorithm 1: P empty -> 0; L = min(C_max, remaining); A empty -> L; B = min_i(d_i) - now; upper-mid

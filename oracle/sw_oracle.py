@@ -283,5 +283,9 @@ class ResidualTable:
                 best = v if best is None else max(best, v)
         return best
 
+    def reset(self) -> None:
+        """Forget every residual (a new cost table makes the old residuals meaningless)."""
+        self.kept = [[[] for _ in self.c_edges] for _ in self.n_edges]
+
     def exceeds(self, n: int, c: int, configured_margin_ns: int, percentile_ppm: int = 990_000, min_samples: int = 1) -> bool:
         return self.margin(n, c, percentile_ppm, min_samples, 0) > configured_margin_ns

@@ -66,7 +66,8 @@ EXPORTS = ["sw_workspace_bytes", "sw_create", "sw_destroy", "sw_kv_append", "sw_
            "sw_mixed_iteration_host", "sw_cost_probe", "sw_cost_probe_iteration", "sw_check_status", "sw_cost_table_create",
            "sw_cost_table_destroy", "sw_cost_table_lookup", "sw_choose_chunk", "sw_choose_chunks", "sw_last_error",
            "sw_decode_attn_static", "sw_selftest_wait_timeout", "sw_telemetry_create", "sw_telemetry_destroy",
-           "sw_telemetry_record", "sw_telemetry_margin", "sw_telemetry_exceeds", "sw_telemetry_get_totals"]
+           "sw_telemetry_record", "sw_telemetry_margin", "sw_telemetry_exceeds", "sw_telemetry_get_totals",
+           "sw_telemetry_reset"]
 
 _vp, _i32, _i64 = C.c_void_p, C.c_int32, C.c_int64
 _lib.sw_workspace_bytes.restype = C.c_size_t
@@ -96,6 +97,7 @@ _lib.sw_telemetry_destroy.restype = None
 _lib.sw_telemetry_record.argtypes = [_vp, _i32, _i32, _i64, _i64, _i64, _i32]
 _lib.sw_telemetry_margin.argtypes = [_vp, _i32, _i32, _i32, _i32, _i64, C.POINTER(_i64)]
 _lib.sw_telemetry_exceeds.argtypes = [_vp, _i32, _i32, _i32, _i32, _i64, C.POINTER(_i32)]
+_lib.sw_telemetry_reset.argtypes = [_vp]
 _lib.sw_telemetry_get_totals.argtypes = [_vp, C.POINTER(sw_telemetry_totals)]
 _lib.sw_cost_table_destroy.restype = None
 _lib.sw_cost_table_lookup.argtypes = [_vp, _i64, _i64, _i64, _i64, C.POINTER(_i64)]
@@ -360,6 +362,9 @@ class Telemetry:
         _check(_lib.sw_telemetry_exceeds(self.handle, n, c, percentile_ppm, min_samples, configured_margin_ns,
                                          C.byref(out)), "sw_telemetry_exceeds")
         return bool(out.value)
+
+    def reset(self) -> None:
+        _check(_lib.sw_telemetry_reset(self.handle), "sw_telemetry_reset")
 
     def totals(self) -> dict:
         t = sw_telemetry_totals()

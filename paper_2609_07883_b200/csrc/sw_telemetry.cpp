@@ -114,6 +114,15 @@ sw_status sw_telemetry_exceeds(const sw_telemetry* t, int32_t n, int32_t c, int3
     return SW_OK;
 }
 
+sw_status sw_telemetry_reset(sw_telemetry* t) {
+    if (!t) return sw_fail(SW_ERR_INVALID_ARG, "sw_telemetry_reset: null argument");
+    for (auto& ring : t->rings) {
+        ring.v.clear();
+        ring.next = 0;
+    }
+    return SW_OK;
+}
+
 sw_status sw_telemetry_get_totals(const sw_telemetry* t, sw_telemetry_totals* out) {
     if (!t || !out) return sw_fail(SW_ERR_INVALID_ARG, "sw_telemetry_get_totals: invalid argument");
     *out = t->totals;

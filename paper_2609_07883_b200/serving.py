@@ -91,7 +91,8 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
               ctx_cap: int | None = None, seed: int = W.SEED_BASE + 44, log=None, page_tables: bool = True,
               ttft_slo_ms: float | None = None, telemetry=None, fallback_margin_ns: int | None = None,
               residual_percentile_ppm: int = 990_000, residual_min_samples: int = 8, fallback_hold: int = 8,
-              max_prefills: int = 1, prefix_cap: int | None = None) -> dict:
+              max_prefills: int = 1, prefix_cap: int | None = None, reprofile=None,
+              reprofile_after_fallbacks: int = 64) -> dict:
     """Run the whole trace; returns statistics.  ``policy`` is "sloweave" or "fixed:<chunk>".  ``execute(batch)`` runs
     one iteration and returns its duration in ns (``gpu_executor`` for the CUDA path).  ``ctx_cap`` clamps the total
     context passed to the table lookup to the table's last grid point.  ``page_tables=False`` hands ``execute`` a batch
@@ -103,6 +104,10 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
     margin, and, when ``fallback_margin_ns`` is given and the residuals exceed it, the iteration runs decode-only.  So
     that a stale residual cannot starve the queue, at most ``fallback_hold`` consecutive iterations fall back; the next
     one admits a chunk again under the residual margin and so refreshes the residuals.
+
+    ``reprofile`` (a callable returning a fresh ``binding.CostTable``) is the re-profiling hook of Sec. 5.1: after
+    ``reprofile_after_fallbacks`` fallback iterations since the last table the loop asks for a new table and starts a
+    new residual window (the telemetry object's old residuals age out of its sliding window).
 
     ``max_prefills > 1`` (SLOWeave policy only) admits several pending prompts per iteration by first fit
     (``sw_choose_chunks``, Sec. 3.3 "Prefill batching"): whole prompts oldest first while the prediction for the total
@@ -130,6 +135,7 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
     misses_chunk = misses_decode_only = infeasible_flags = stalled_for_memory = 0
     chunks, iter_ns, pred_err = [], [], []
     fallback_iters = fallback_run = 0
+    fallbacks_since_table = reprofiles = 0
     prompts_per_chunk_iter = []
     prefill_tokens = 0
     wall0 = time.time()
@@ -174,6 +180,12 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
             c = 0
             fallback_run += 1
             fallback_iters += 1
+            fallbacks_since_table += 1
+            if reprofile is not None and fallbacks_since_table >= reprofile_after_fallbacks:
+                table = reprofile()
+                telemetry.reset()          # residuals against the old table say nothing about the new one
+                reprofiles += 1
+                fallbacks_since_table = 0
         elif fixed_chunk is not None:
             c = min(fixed_chunk, remaining)
         elif max_prefills > 1 and head is not None:
@@ -318,7 +330,7 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
         "tpot_ms_p99_of_request_p99": float(np.percentile(p99_gap, 99)),
         "requests_meeting_tpot": int(np.sum(p99_gap <= tpot_each)),
         "prediction_error_ms_p99": float(np.percentile(pred_err, 99)) / MS if pred_err else 0.0,
-        "fallback_iterations": fallback_iters,
+        "fallback_iterations": fallback_iters, "reprofiles": reprofiles,
         "mean_prompts_per_chunk_iteration": float(np.mean(prompts_per_chunk_iter)) if prompts_per_chunk_iter else 0.0,
         "margin_ppm": margin_ppm, "c_max": c_max, "quantum": quantum, "wall_s": time.time() - wall0,
     }

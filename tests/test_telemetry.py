@@ -29,6 +29,9 @@ def test_margins_match_the_oracle_on_random_streams(B, oracle):
             pred, obs = int(rng.integers(0, 10**7)), int(rng.integers(0, 10**7))
             lib_t.record(n, c, pred, obs, slack_ns=int(rng.integers(-5, 5)), fallback=bool(step % 7 == 0))
             ref_t.record(n, c, pred, obs)
+            if step == 250 and trial % 2:
+                lib_t.reset()
+                ref_t.reset()
             if step % 9 == 0:
                 qn, qc = int(rng.integers(0, 700)), int(rng.integers(0, 6000))
                 ppm = int(rng.choice([1, 500_000, 900_000, 990_000, 1_000_000]))
@@ -89,3 +92,35 @@ def test_feedback_loop_absorbs_an_under_predicting_table(B, oracle):
     strict = serving.run_trace(trace, 10.0, table, slow, telemetry=tel2, fallback_margin_ns=200_000, **kw)
     assert strict["fallback_iterations"] > 0
     assert strict["prefill_tokens"] == int(trace["prompt_len"].sum())
+
+
+def test_reprofiling_hook_replaces_a_stale_table(B, oracle):
+    """Sec. 5.1: when the residuals keep exceeding the configured margin the runtime measures a new table.  Here the
+    executor is 12 % slower than the first table; the hook returns a table of the slower machine, after which the
+    fallback stops firing."""
+    from paper_2609_07883_b200 import serving
+
+    n_values = list(range(1, 129))
+    chunk_grid = list(range(0, 2049, 16))
+    cost = np.array([[oracle.analytic_cost_ns(n, c) for c in chunk_grid] for n in n_values], dtype=np.int64)
+    stale = B.CostTable(n_values, [1 << 40], [1 << 30], chunk_grid, cost.reshape(len(n_values), 1, 1, -1))
+    fresh_cost = (cost * 1.12).astype(np.int64) + 1
+    calls = []
+
+    def reprofile():
+        calls.append(1)
+        return B.CostTable(n_values, [1 << 40], [1 << 30], chunk_grid, fresh_cost.reshape(len(n_values), 1, 1, -1))
+
+    trace = W.bursty_trace(num_requests=300, rate_low=30.0, rate_high=90.0, mean_dwell_s=1.0, prompt_median=1500.0,
+                           prompt_clip=(32, 4096), mean_output=60.0, rng=np.random.default_rng(9))
+    slow = lambda batch: int(oracle.analytic_cost_ns(batch.num_decode, batch.chunk_len) * 1.12)
+    kw = dict(shape=W.LLAMA, num_pages=1 << 16, policy="sloweave", c_max=2048, margin_ppm=0, quantum=16, max_decode=128,
+              page_tables=False, fallback_margin_ns=200_000)
+    tel = B.Telemetry([4, 16, 64, 128], [0, 256, 1024, 2048], window=32)
+    without = serving.run_trace(trace, 10.0, stale, slow, telemetry=B.Telemetry([4, 16, 64, 128], [0, 256, 1024, 2048], window=32),
+                                **kw)
+    with_hook = serving.run_trace(trace, 10.0, stale, slow, telemetry=tel, reprofile=reprofile, reprofile_after_fallbacks=32,
+                                  **kw)
+    assert len(calls) == with_hook["reprofiles"] >= 1
+    assert with_hook["fallback_iterations"] < without["fallback_iterations"] // 4
+    assert with_hook["prefill_tokens"] == int(trace["prompt_len"].sum())
