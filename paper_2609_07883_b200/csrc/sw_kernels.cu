@@ -30,8 +30,11 @@ __device__ __forceinline__ void report(int32_t* ctrl, int code, int site, int in
 // ---------------------------------------------------------------------------------------------------------------
 // One thread per (row, 16-byte piece of the row's Hkv*D elements); it copies that piece of K and of V.  `first` and
 // `stride` spread the pieces over the calling threads.
-__device__ __forceinline__ void append_rows(const AppendParams& p, int64_t first, int64_t stride) {
-    const int pieces_per_row = p.Hkv * p.D / 8;
+// (P is AppendParams or MixedParams: the fields have the same names; every index into the chunk arrays is a
+// compile-time constant so that the kernel parameters stay in constant memory.)
+template <bool kMulti, class P>
+__device__ __forceinline__ void append_rows(const P& p, int head_dim, int64_t first, int64_t stride) {
+    const int pieces_per_row = p.Hkv * head_dim / 8;
     const int64_t total = (int64_t)(p.C + p.n) * pieces_per_row;
     for (int64_t idx = first; idx < total; idx += stride) {
         const int row = (int)(idx / pieces_per_row);
@@ -40,11 +43,19 @@ __device__ __forceinline__ void append_rows(const AppendParams& p, int64_t first
         const int32_t* pages;
         int npages;
         if (row < p.C) {
-            int j = 0;  // the chunk this row belongs to
-            while (j + 1 < p.nchunks && row >= p.cRow0[j + 1]) ++j;
-            pos = (int64_t)p.cP[j] + (row - p.cRow0[j]);
-            pages = p.prefill_pages + p.cPage0[j];
-            npages = p.cPage0[j + 1] - p.cPage0[j];
+            // the chunk this row belongs to: the last one that starts at or before it
+            int cP = p.cP[0], cRow0 = 0, page0 = 0, page1 = p.num_prefill_pages;
+#pragma unroll
+            for (int j = 0; j < kMaxChunks; ++j)
+                if (kMulti && j < p.nchunks && row >= p.cRow0[j]) {
+                    cP = p.cP[j];
+                    cRow0 = p.cRow0[j];
+                    page0 = p.cPage0[j];
+                    page1 = p.cPage0[j + 1];
+                }
+            pos = (int64_t)cP + (row - cRow0);
+            pages = p.prefill_pages + page0;
+            npages = page1 - page0;
         } else {
             const int i = row - p.C;
             const int len = p.decode_kv_len[i];
@@ -69,11 +80,11 @@ __device__ __forceinline__ void append_rows(const AppendParams& p, int64_t first
             continue;
         }
         const int e0 = piece * 8;          // element offset inside the row's [Hkv][D]
-        const int kvh = e0 / p.D;
-        const int e = e0 % p.D;
-        const int64_t src = (int64_t)row * p.Hkv * p.D + e0;
-        const int64_t dst_k = ((((int64_t)page * 2 + 0) * p.Hkv + kvh) * kPageSize + slot) * p.D + e;
-        const int64_t dst_v = ((((int64_t)page * 2 + 1) * p.Hkv + kvh) * kPageSize + slot) * p.D + e;
+        const int kvh = e0 / head_dim;
+        const int e = e0 % head_dim;
+        const int64_t src = (int64_t)row * p.Hkv * head_dim + e0;
+        const int64_t dst_k = ((((int64_t)page * 2 + 0) * p.Hkv + kvh) * kPageSize + slot) * head_dim + e;
+        const int64_t dst_v = ((((int64_t)page * 2 + 1) * p.Hkv + kvh) * kPageSize + slot) * head_dim + e;
         *reinterpret_cast<uint4*>(p.pool + dst_k) = *reinterpret_cast<const uint4*>(p.k_new + src);
         *reinterpret_cast<uint4*>(p.pool + dst_v) = *reinterpret_cast<const uint4*>(p.v_new + src);
     }
@@ -84,7 +95,7 @@ __global__ void sw_kv_append_kernel(const AppendParams p) {
     // the previous iteration, possibly still reading this pool) drains; nothing is touched before this wait
     grid_launch_dependents();
     grid_dependency_wait();
-    append_rows(p, (int64_t)blockIdx.x * blockDim.x + threadIdx.x, (int64_t)gridDim.x * blockDim.x);
+    append_rows<true>(p, p.D, (int64_t)blockIdx.x * blockDim.x + threadIdx.x, (int64_t)gridDim.x * blockDim.x);
 }
 
 cudaError_t launch_kv_append(const AppendParams& p, cudaStream_t stream) {
@@ -734,7 +745,7 @@ namespace sw {
 // ---------------------------------------------------------------------------------------------------------------
 // the persistent kernel
 // ---------------------------------------------------------------------------------------------------------------
-template <int D>
+template <int D, bool kMulti>
 __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid_constant__ CUtensorMap kv_map,
                                                                        const __grid_constant__ CUtensorMap kvp_map,
                                                                     const __grid_constant__ CUtensorMap q_map,
@@ -752,6 +763,18 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     const bool tensor_prefill = p.C > 0;
     volatile int* misc = reinterpret_cast<volatile int*>(scratch + 32);  // [0] TMEM base, [1] abort flag, [2..3] ticket flags
     if (threadIdx.x >= 32 && threadIdx.x < 32 + kPlanCounters) scratch[64 + threadIdx.x - 32] = 0;  // block-sum counters
+    // the chunks' descriptors go to shared memory: the roles of the chunk-prefill phase look them up by the item's chunk
+    // number instead of carrying them in registers
+    if (kMulti && threadIdx.x == 64) {
+        int* tbl = scratch + kChunkTable;
+#pragma unroll
+        for (int j = 0; j < kMaxChunks; ++j) {
+            tbl[j] = p.cP[j];
+            tbl[kMaxChunks + j] = p.cC[j];
+            tbl[2 * kMaxChunks + j] = p.cRow0[j];
+            tbl[3 * kMaxChunks + j] = p.cPage0[j];
+        }
+    }
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&kv_map);
         tma_prefetch_desc(&kvp_map);
@@ -770,30 +793,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     grid_launch_dependents();
     if (p.pool != nullptr) {
         // fused launch: this CTA's share of the new K/V rows, then its mark on the counter the readers wait for
-        AppendParams a;
-        a.Hkv = p.Hkv;
-        a.D = D;
-        a.num_pages = p.num_pages;
-        a.C = p.C;
-        a.n = p.n;
-        a.nchunks = p.nchunks;
-        for (int j = 0; j < kMaxChunks; ++j) {
-            a.cP[j] = p.cP[j];
-            a.cC[j] = p.cC[j];
-            a.cRow0[j] = p.cRow0[j];
-            a.cPage0[j] = p.cPage0[j];
-        }
-        a.cPage0[kMaxChunks] = p.cPage0[kMaxChunks];
-        a.prefill_pages = p.prefill_pages;
-        a.num_prefill_pages = p.num_prefill_pages;
-        a.decode_kv_len = p.decode_kv_len;
-        a.decode_page_indptr = p.decode_page_indptr;
-        a.decode_pages = p.decode_pages;
-        a.k_new = p.k_new;
-        a.v_new = p.v_new;
-        a.pool = p.pool;
-        a.ctrl = p.ctrl;
-        append_rows(a, (int64_t)blockIdx.x * kThreads + threadIdx.x, (int64_t)gridDim.x * kThreads);
+        append_rows<kMulti>(p, D, (int64_t)blockIdx.x * kThreads + threadIdx.x, (int64_t)gridDim.x * kThreads);
         fence_proxy_async_global();
         __threadfence();
         __syncthreads();
@@ -807,7 +807,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     int prefill_ctas = 0;
     LateJoin late{0, 0.f};
     if (tensor_prefill) {
-        const PfPlan pplan = pf_make_plan(p);
+        const PfPlan pplan = pf_make_plan<kMulti>(p);
         prefill_ctas = min(pplan.n_entries, (int)gridDim.x);
         late.ctas = prefill_ctas;
         late.us = kLateBaseUs + kLateStepUs * ((pplan.longest + pplan.pieces - 1) / pplan.pieces);
@@ -830,7 +830,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
             scr.o = p.pf_o;
             scr.tickets = p.pf_tickets;
             scr.flags = &misc[2];
-            prefill_phase<D>(&kv_map, &q_map, p, sh, pplan, scr, first_entry, &misc[5]);
+            prefill_phase<D, kMulti>(&kv_map, &q_map, p, sh, pplan, scr, first_entry, &misc[5]);
             tc_fence_before_sync();
             __syncthreads();
             if (warp == 1) tmem_dealloc(sh.tmem, 512);
@@ -934,12 +934,19 @@ size_t mixed_attn_smem_bytes(int head_dim) {
     return (head_dim == 64 ? Geo<64>::kSmemBytes : Geo<128>::kSmemBytes) + 1024;
 }
 
+// The kernel exists in two forms per head size: for iterations with at most one prefill chunk, whose descriptors are
+// then plain kernel parameters, and for iterations with several (descriptors looked up per work item).
 cudaError_t configure_kernels(int head_dim) {
-    if (head_dim == 64)
-        return cudaFuncSetAttribute(sw_mixed_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)mixed_attn_smem_bytes(64));
-    return cudaFuncSetAttribute(sw_mixed_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)mixed_attn_smem_bytes(128));
+    const int bytes = (int)mixed_attn_smem_bytes(head_dim);
+    cudaError_t e;
+    if (head_dim == 64) {
+        e = cudaFuncSetAttribute(sw_mixed_attn_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e != cudaSuccess) return e;
+        return cudaFuncSetAttribute(sw_mixed_attn_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    }
+    e = cudaFuncSetAttribute(sw_mixed_attn_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(sw_mixed_attn_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
 }
 
 cudaError_t launch_mixed_attn(int head_dim, const KvMaps& kv_maps, const CUtensorMap& q_map, const MixedParams& p,
@@ -954,8 +961,12 @@ cudaError_t launch_mixed_attn(int head_dim, const KvMaps& kv_maps, const CUtenso
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (head_dim == 64) return cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<64>, kv_maps.tile, kv_maps.page, q_map, p);
-    return cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<128>, kv_maps.tile, kv_maps.page, q_map, p);
+    const bool multi = p.nchunks > 1;
+    if (head_dim == 64)
+        return multi ? cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<64, true>, kv_maps.tile, kv_maps.page, q_map, p)
+                     : cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<64, false>, kv_maps.tile, kv_maps.page, q_map, p);
+    return multi ? cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<128, true>, kv_maps.tile, kv_maps.page, q_map, p)
+                 : cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<128, false>, kv_maps.tile, kv_maps.page, q_map, p);
 }
 
 }  // namespace sw

@@ -34,12 +34,27 @@ enum PfBar {
 // register budgets per warpgroup during the prefill phase: 128 * 72 + 256 * 216 <= 384 * 168
 constexpr int kPfRegsLaunch = 168, kPfRegsLight = 72, kPfRegsHeavy = 216;
 
+constexpr int kChunkTable = 88;  // ints into the CTA's scratch: P[8], C[8], first row[8], page-list offset[8] of the chunks
+
 struct PfShared {
     uint32_t smem;    // 1024-aligned shared address of the tile region
     uint32_t bars;    // shared address of the kPfBars mbarriers
     uint32_t tmem;    // TMEM base (lane 0, column 0 of the 512-column allocation)
     volatile int* abort_flag;
 };
+
+// Field `field` (0 prefix length, 1 tokens, 2 first row, 3 page-list offset) of chunk `chunk` from the table in shared
+// memory; its address follows from the tile region's, so no role keeps a pointer to it.
+// A kernel that serves a single chunk (kMulti = false) reads the kernel parameters instead, which costs no register
+// and no instruction in any role.
+template <int D, bool kMulti>
+__device__ __forceinline__ int pf_chunk(const MixedParams& p, const PfShared& sh, int field, int chunk) {
+    if constexpr (!kMulti) {
+        return field == 0 ? p.cP[0] : (field == 1 ? p.cC[0] : 0);
+    } else {
+        return lds_s32(sh.smem + Geo<D>::kMiscOffset + (kChunkTable + field * kMaxChunks + chunk) * 4);
+    }
+}
 
 __device__ __forceinline__ void pf_init_barriers(uint32_t bars) {
     for (int i = 0; i < kPfBars; ++i) mbar_init(bars + i * 8, (i >= kBarPHalf && i < kBarPHalf + 4) ? 4 : 1);
@@ -75,8 +90,7 @@ __device__ __forceinline__ bool pf_wait(const PfShared& sh, int bar, uint32_t pa
 constexpr int kPfMinPieceSteps = SW_PF_MIN_PIECE_STEPS;
 
 struct PfPlan {
-    int items_before[kMaxChunks + 1];  // items of the chunks before chunk j (items are numbered chunk by chunk)
-    int longest, shortest;             // steps of the longest and of the shortest item
+    int longest, shortest;             // steps of the longest and of the shortest item (items are numbered chunk by chunk)
     int n_items;        // sum over chunks of (256-row groups) * Hkv
     int n_whole;        // entries [0, n_whole) are whole items
     int pieces;         // k: pieces per tail item (1 = tail items are whole too)
@@ -87,9 +101,7 @@ struct PfPlan {
 struct PfItem {
     int item;        // number of the item among all chunks' items; within its chunk: rank * Hkv + kvh
     int kvh;
-    int P, C;        // the chunk's prefix length and tokens
-    int row0;        // the chunk's first row of q / out
-    const int32_t* pages;  // the page list of the chunk's prompt
+    int chunk;       // which chunk of the iteration the item belongs to (its descriptors are in the shared table)
     int tok0[2];     // first chunk token of each tile
     int nkv[2];      // KV tiles each tile attends in total (0 = tile has no rows)
     int nk;          // steps of the item = max(nkv)
@@ -116,6 +128,7 @@ __device__ __forceinline__ int pf_steps_of_rank(int group, int P, int C, int n_t
 // first KV tile of piece i when nk steps are cut into k pieces
 __device__ __forceinline__ int pf_piece_begin(int nk, int k, int i) { return (int)(((long long)nk * i) / k); }
 
+template <bool kMulti>
 __device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p) {
     PfPlan plan;
     const int G = (int)gridDim.x;
@@ -124,8 +137,7 @@ __device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p) {
     plan.shortest = 0x7fffffff;
 #pragma unroll
     for (int j = 0; j < kMaxChunks; ++j) {
-        plan.items_before[j] = plan.n_items;
-        if (j < p.nchunks) {
+        if (j < (kMulti ? p.nchunks : 1)) {
             const int n_tp = pf_num_groups(p.group, p.cC[j]);
             plan.n_items += n_tp * p.Hkv;
             if (n_tp > 0) {
@@ -134,7 +146,6 @@ __device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p) {
             }
         }
     }
-    plan.items_before[kMaxChunks] = plan.n_items;
     const int r = plan.n_items % G;
     plan.n_whole = plan.n_items - r;
     plan.pieces = 1;
@@ -153,6 +164,7 @@ __device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p) {
     return plan;
 }
 
+template <bool kMulti>
 __device__ __forceinline__ PfItem pf_entry(const MixedParams& p, const PfPlan& plan, int entry) {
     PfItem it;
     if (entry < plan.n_whole) {
@@ -162,22 +174,30 @@ __device__ __forceinline__ PfItem pf_entry(const MixedParams& p, const PfPlan& p
         it.item = plan.n_whole + (entry - plan.n_whole) / plan.pieces;
         it.piece = (entry - plan.n_whole) % plan.pieces;
     }
-    int chunk = 0;
+    // the item's chunk: the last one whose items start at or before it.  The chunks' item counts are recomputed here
+    // (a table of them would sit in registers of every role for the whole phase); indices into the kernel parameters
+    // are compile-time constants so that the parameters stay in constant memory.
+    int before = 0, count = 0, cP = p.cP[0], cC = p.cC[0];
+    it.chunk = 0;
 #pragma unroll
-    for (int j = 1; j < kMaxChunks; ++j)
-        if (j < p.nchunks && it.item >= plan.items_before[j]) chunk = j;
-    it.P = p.cP[chunk];
-    it.C = p.cC[chunk];
-    it.row0 = p.cRow0[chunk];
-    it.pages = p.prefill_pages + p.cPage0[chunk];
-    const int local = it.item - plan.items_before[chunk];
+    for (int j = 0; j < kMaxChunks; ++j)
+        if (kMulti && j < p.nchunks) {
+            if (it.item >= count) {
+                before = count;
+                it.chunk = j;
+                cP = p.cP[j];
+                cC = p.cC[j];
+            }
+            count += pf_num_groups(p.group, p.cC[j]) * p.Hkv;
+        }
+    const int local = it.item - before;
     const int rank = local / p.Hkv;
     it.kvh = local % p.Hkv;
     const int tt = 128 / p.group;
-    const int tp = pf_num_groups(p.group, it.C) - 1 - rank;
+    const int tp = pf_num_groups(p.group, cC) - 1 - rank;
     for (int t = 0; t < 2; ++t) {
         it.tok0[t] = (tp * 2 + t) * tt;
-        it.nkv[t] = pf_tiles_of(p.group, it.P, it.C, it.tok0[t]);
+        it.nkv[t] = pf_tiles_of(p.group, cP, cC, it.tok0[t]);
     }
     it.nk = max(it.nkv[0], it.nkv[1]);
     if (entry < plan.n_whole) {
@@ -193,7 +213,7 @@ __device__ __forceinline__ PfItem pf_entry(const MixedParams& p, const PfPlan& p
 }
 
 // ---- role: TMA producer (one warp) ----------------------------------------------------------------------------
-template <int D>
+template <int D, bool kMulti>
 __device__ __forceinline__ bool pf_produce(const CUtensorMap* kv_map, const CUtensorMap* q_map, const MixedParams& p,
                                            const PfShared& sh, const PfItem& it, uint32_t& kv_it) {
     using G = PfGeo<D>;
@@ -208,18 +228,20 @@ __device__ __forceinline__ bool pf_produce(const CUtensorMap* kv_map, const CUte
             if (it.nkv[t] > it.j0)
                 for (int h = 0; h < G::kHalves; ++h)
                     tma_load_3d(sh.smem + G::kQOffset + t * G::kTileBytes + h * G::kHalfBytes, q_map, sh.bars + kBarQFull * 8,
-                                h * 64, it.kvh * p.group, it.row0 + it.tok0[t]);
+                                h * 64, it.kvh * p.group, pf_chunk<D, kMulti>(p, sh, 2, it.chunk) + it.tok0[t]);
     }
     // fused launch: tiles that reach into the chunk's own keys wait until every CTA has written its share of them
-    if (p.pool != nullptr && it.j1 * 128 > it.P && !wait_append(p)) {
+    if (p.pool != nullptr && it.j1 * 128 > pf_chunk<D, kMulti>(p, sh, 0, it.chunk) && !wait_append(p)) {
         if (lane == 0) {
             *sh.abort_flag = 1;
             report(p.ctrl, SW_ERR_DEVICE_TIMEOUT, kSiteWait, it.item);
         }
         return false;
     }
-    const int npages = (it.P + it.C + kPageSize - 1) / kPageSize;
-    auto page_of = [&](int j) { return (lane < 8 && j * 8 + lane < npages) ? it.pages[j * 8 + lane] : 0; };
+    const int npages = (pf_chunk<D, kMulti>(p, sh, 0, it.chunk) + pf_chunk<D, kMulti>(p, sh, 1, it.chunk) + kPageSize - 1) / kPageSize;
+    auto page_of = [&](int j) {
+        return (lane < 8 && j * 8 + lane < npages) ? p.prefill_pages[pf_chunk<D, kMulti>(p, sh, 3, it.chunk) + j * 8 + lane] : 0;
+    };
     int id_next = page_of(it.j0);
     for (int j = it.j0; j < it.j1; ++j, ++kv_it) {
         const uint32_t s = kv_it & 1, n = kv_it >> 1;
@@ -249,11 +271,11 @@ __device__ __forceinline__ bool pf_produce(const CUtensorMap* kv_map, const CUte
 // ---- role: V sanitizer (one warp) -------------------------------------------------------------------------------
 // Keys at or past P + C are never attended, but their V rows still enter the P V product with weight zero; zero them
 // so that whatever an unwritten page slot (or a stale buffer) holds cannot turn 0 * x into NaN.
-template <int D>
+template <int D, bool kMulti>
 __device__ __forceinline__ bool pf_sanitize(const MixedParams& p, const PfShared& sh, const PfItem& it, uint32_t& kv_it) {
     using G = PfGeo<D>;
     const int lane = threadIdx.x & 31;
-    const int kv_total = it.P + it.C;
+    const int kv_total = pf_chunk<D, kMulti>(p, sh, 0, it.chunk) + pf_chunk<D, kMulti>(p, sh, 1, it.chunk);
     for (int j = it.j0; j < it.j1; ++j, ++kv_it) {
         const uint32_t s = kv_it & 1, n = kv_it >> 1;
         if (!pf_wait(sh, kBarVLanded + s, n & 1, p.ctrl, 3)) return false;
@@ -408,7 +430,7 @@ struct PfScratch {
     volatile int* flags;  // shared memory, one int per tile: ticket value seen by the warpgroup's thread 0
 };
 
-template <int D>
+template <int D, bool kMulti>
 __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared& sh, const PfPlan& plan,
                                            const PfScratch& scr, const PfItem& it, int t, PfSoftmaxState& st) {
     if (it.j1 <= it.j0) return true;  // an empty piece (more pieces than steps)
@@ -418,7 +440,7 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
     const int row = (warp & 3) * 32 + lane;
     const int tok = it.tok0[t] + row / p.group;
     const int head = it.kvh * p.group + row % p.group;
-    const int pos = it.P + tok;
+    const int pos = pf_chunk<D, kMulti>(p, sh, 0, it.chunk) + tok;
     const uint32_t lane_addr = sh.tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t s_addr = lane_addr + t * 128;  // P (bf16) aliases the first 64 columns of S
     const uint32_t o_addr = lane_addr + 256 + t * D;
@@ -525,8 +547,8 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
     if (!pf_wait(sh, kBarODone + t, (st.o_cnt + (j_end - it.j0) - 1) & 1, p.ctrl, 11)) return false;
     st.o_cnt += j_end - it.j0;
     tc_fence_after_sync();
-    const bool row_ok = tok < it.C;
-    const int64_t out_row = (int64_t)it.row0 + tok;
+    const bool row_ok = tok < pf_chunk<D, kMulti>(p, sh, 1, it.chunk);
+    const int64_t out_row = (int64_t)pf_chunk<D, kMulti>(p, sh, 2, it.chunk) + tok;
     __nv_bfloat16* dst = p.out + (out_row * p.Hq + head) * D;
     const bool whole = it.j0 == 0 && j_end == it.nkv[t];  // this piece holds every step of the tile
     if (whole) {
@@ -638,7 +660,7 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
 // ---- the prefill phase of one CTA ----------------------------------------------------------------------------------
 // `next` points at two shared-memory ints: the idle warp fetches the following entry from the global counter while
 // the current one is processed and leaves it in next[iteration parity]; everyone reads it after the piece barrier.
-template <int D>
+template <int D, bool kMulti>
 __device__ __forceinline__ void prefill_phase(const CUtensorMap* kv_map, const CUtensorMap* q_map, const MixedParams& p,
                                               const PfShared& sh, const PfPlan& plan, const PfScratch& scr, int first_entry,
                                               volatile int* next) {
@@ -661,13 +683,13 @@ __device__ __forceinline__ void prefill_phase(const CUtensorMap* kv_map, const C
         setmaxnreg_dec<kPfRegsLight>();
         int entry = first_entry;
         for (int iter = 0; entry < plan.n_entries; ++iter) {
-            const PfItem it = pf_entry(p, plan, entry);
+            const PfItem it = pf_entry<kMulti>(p, plan, entry);
             if (warp == 0) {
-                if (it.j1 > it.j0) pf_produce<D>(kv_map, q_map, p, sh, it, prod_kv_it);
+                if (it.j1 > it.j0) pf_produce<D, kMulti>(kv_map, q_map, p, sh, it, prod_kv_it);
             } else if (warp == 1) {
                 if (it.j1 > it.j0) pf_mma<D>(p, sh, it, mma_state);
             } else if (warp == 2) {
-                if (it.j1 > it.j0) pf_sanitize<D>(p, sh, it, san_kv_it);
+                if (it.j1 > it.j0) pf_sanitize<D, kMulti>(p, sh, it, san_kv_it);
             } else {
                 // entries 0 .. gridDim.x-1 are the CTAs' first ones; the counter hands out the rest
                 if (lane == 0) next[iter & 1] = (int)gridDim.x + atomicAdd(&p.ctrl[kCtrPrefill], 1);
@@ -680,8 +702,8 @@ __device__ __forceinline__ void prefill_phase(const CUtensorMap* kv_map, const C
         setmaxnreg_inc<kPfRegsHeavy>();
         int entry = first_entry;
         for (int iter = 0; entry < plan.n_entries; ++iter) {
-            const PfItem it = pf_entry(p, plan, entry);
-            pf_softmax<D>(p, sh, plan, scr, it, (warp - 4) >> 2, sm_state);
+            const PfItem it = pf_entry<kMulti>(p, plan, entry);
+            pf_softmax<D, kMulti>(p, sh, plan, scr, it, (warp - 4) >> 2, sm_state);
             if (!piece_sync()) break;
             entry = next[iter & 1];
         }

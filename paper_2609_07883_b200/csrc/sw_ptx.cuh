@@ -65,6 +65,12 @@ __device__ __forceinline__ int ld_acquire_gpu(const int* ptr) {
     return v;
 }
 
+__device__ __forceinline__ int lds_s32(uint32_t addr) {
+    int v;
+    asm volatile("ld.shared.s32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+
 // ---- TMA tiled loads / stores (no multicast anywhere) ---------------------------------------------------------
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
