@@ -365,7 +365,7 @@ def run_ours(args) -> dict:
         "attn_launch_us": attn_ms * 1e3,
         "roofline": {"bound": "hbm", "achieved": achieved_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved_gbs / peaks["hbm_gbs"], "traffic": traffic, "peak_kind": f"of {peak_kind}",
-                     "kernel": "sw_mixed_attn_kernel<128> (KV append fused in)", "algorithmic_bytes_per_launch": launch_bytes,
+                     "kernel": "sw_mixed_attn_kernel<128, false> (one prefill chunk; KV append fused in)", "algorithmic_bytes_per_launch": launch_bytes,
                      "attention_only_launch_gbs": work["attn_bytes"] / (attn_ms * 1e-3) / 1e9,
                      "frac_of_nominal_8TBs": achieved_gbs / NOMINAL_HBM_GBS,
                      "prefill_tflops": work["prefill_flops"] / (us * 1e-6) / 1e12},
