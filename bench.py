@@ -324,8 +324,9 @@ def run_ours(args) -> dict:
     hs, keep = B.host_batch_struct(batch)
     h_q, h_k, h_v = (t.cpu().pin_memory() for t in (q, k_new, v_new))
     h_out = torch.empty_like(h_q).pin_memory()
-    e2e_steps = max(3, min(args.steps, 20))
-    for i in range(2):
+    # (the first hundred or so calls run slower than the steady state: pinned-copy paths and clocks settle)
+    e2e_steps = max(3, min(args.steps, 200))
+    for i in range(max(2, min(args.steps, 100))):
         B.sw_mixed_iteration_host(ctx, pools[i % args.layers], hs, h_q, h_k, h_v, h_out)
     sync_all()
     t0 = time.perf_counter()
