@@ -47,7 +47,8 @@ WsLayout ws_layout(const sw_layout& l, int max_chunk, int max_decode, int64_t ma
     w.tickets = off;  off = align_up(off + (size_t)std::max(1, max_decode) * l.num_kv_heads * 4 * 2, 256);  // tickets, ready
     w.part_ml = off;  off = align_up(off + (size_t)w.max_items * 2 * sw::kMaxGroup * 4, 256);
     w.part_o = off;   off = align_up(off + (size_t)w.max_items * g * l.head_dim * 4, 256);
-    const size_t groups = ((size_t)max_chunk + (256 / g) - 1) / (256 / g);
+    // 256-row groups of the chunks of one iteration: every chunk may end in a ragged group
+    const size_t groups = ((size_t)max_chunk + (256 / g) - 1) / (256 / g) + sw::kMaxChunks;
     w.pf_tickets = off; off = align_up(off + std::max<size_t>(1, groups) * l.num_kv_heads * 2 * 4, 256);
     w.pf_ml = off;    off = align_up(off + (size_t)sw::kMaxCtas * 2 * 256 * 4, 256);
     w.pf_o = off;     off = align_up(off + (max_chunk > 0 ? (size_t)sw::kMaxCtas * 2 * 128 * l.head_dim * 4 : 0), 256);

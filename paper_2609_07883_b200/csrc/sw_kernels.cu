@@ -157,7 +157,7 @@ struct Geo {
     static constexpr int kLenOffset = kPlanOffset + (kMaxDecode + 1) * 4 + 12;  // int32 kv_len[kMaxDecode]
     static constexpr int kIndptrOffset = kLenOffset + kMaxDecode * 4;           // int32 page_indptr[kMaxDecode+1]
     static constexpr int kMiscOffset = kIndptrOffset + (kMaxDecode + 1) * 4 + 12; // scan scratch, TMEM base, abort flag
-    static constexpr int kSmemBytes = kMiscOffset + 512;   // 64 ints scan scratch and flags, then the plan's counter
+    static constexpr int kSmemBytes = kMiscOffset + 768;   // 64 ints scan scratch and flags, the plan's counters, the chunk table
 };
 
 constexpr int kOneRoundMaxPages = 48;  // longest unit (pages) for which one round of units is planned
@@ -765,16 +765,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     if (threadIdx.x >= 32 && threadIdx.x < 32 + kPlanCounters) scratch[64 + threadIdx.x - 32] = 0;  // block-sum counters
     // the chunks' descriptors go to shared memory: the roles of the chunk-prefill phase look them up by the item's chunk
     // number instead of carrying them in registers
-    if (kMulti && threadIdx.x == 64) {
-        int* tbl = scratch + kChunkTable;
-#pragma unroll
-        for (int j = 0; j < kMaxChunks; ++j) {
-            tbl[j] = p.cP[j];
-            tbl[kMaxChunks + j] = p.cC[j];
-            tbl[2 * kMaxChunks + j] = p.cRow0[j];
-            tbl[3 * kMaxChunks + j] = p.cPage0[j];
-        }
-    }
+    if (kMulti && warp == 2) pf_fill_chunk_table(p, scratch + kChunkTable);
     if (threadIdx.x == 0) {
         tma_prefetch_desc(&kv_map);
         tma_prefetch_desc(&kvp_map);
@@ -807,7 +798,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     int prefill_ctas = 0;
     LateJoin late{0, 0.f};
     if (tensor_prefill) {
-        const PfPlan pplan = pf_make_plan<kMulti>(p);
+        const PfPlan pplan = pf_make_plan<kMulti>(p, base + Geo<D>::kMiscOffset + kChunkTable * 4);
         prefill_ctas = min(pplan.n_entries, (int)gridDim.x);
         late.ctas = prefill_ctas;
         late.us = kLateBaseUs + kLateStepUs * ((pplan.longest + pplan.pieces - 1) / pplan.pieces);

@@ -34,7 +34,8 @@ enum PfBar {
 // register budgets per warpgroup during the prefill phase: 128 * 72 + 256 * 216 <= 384 * 168
 constexpr int kPfRegsLaunch = 168, kPfRegsLight = 72, kPfRegsHeavy = 216;
 
-constexpr int kChunkTable = 88;  // ints into the CTA's scratch: P[8], C[8], first row[8], page-list offset[8] of the chunks
+constexpr int kChunkTable = 88;  // ints into the CTA's scratch: P[8], C[8], first row[8], page-list offset[8], pieces[8] of the chunks
+constexpr int kChunkTotals = 7 * 8;  // ints into the table: the plan's totals, after seven fields of eight chunks
 
 struct PfShared {
     uint32_t smem;    // 1024-aligned shared address of the tile region
@@ -43,7 +44,7 @@ struct PfShared {
     volatile int* abort_flag;
 };
 
-// Field `field` (0 prefix length, 1 tokens, 2 first row, 3 page-list offset) of chunk `chunk` from the table in shared
+// Field `field` (0 prefix length, 1 tokens, 2 first row, 3 page-list offset, 4 pieces per tail item) of chunk `chunk` from the table in shared
 // memory; its address follows from the tile region's, so no role keeps a pointer to it.
 // A kernel that serves a single chunk (kMulti = false) reads the kernel parameters instead, which costs no register
 // and no instruction in any role.
@@ -93,9 +94,9 @@ struct PfPlan {
     int longest, shortest;             // steps of the longest and of the shortest item (items are numbered chunk by chunk)
     int n_items;        // sum over chunks of (256-row groups) * Hkv
     int n_whole;        // entries [0, n_whole) are whole items
-    int pieces;         // k: pieces per tail item (1 = tail items are whole too)
-    int n_entries;      // n_whole + (n_items - n_whole) * k
-    const int* prefix;  // shared memory [n_tp + 1]: steps of one kv head's items before rank r
+    int pieces;         // k: pieces per tail item (1 = tail items are whole too); several chunks: of the first chunk's
+    int n_entries;      // n_whole + (n_items - n_whole) * k; several chunks: every chunk's tail items times its own k
+    uint32_t table;     // several chunks: shared address of the chunk table (k of chunk j is field 4)
 };
 
 struct PfItem {
@@ -108,6 +109,7 @@ struct PfItem {
     int j0, j1;      // this entry's piece of the item: KV tiles [j0, j1)
     int piece;       // index of the piece (0 when the item is whole)
     int slot0;       // scratch slot of the item's piece 0 (tail items only)
+    int pieces;      // pieces the item is cut into (several chunks: each chunk has its own count)
 };
 
 __device__ __forceinline__ int pf_tiles_of(int group, int P, int C, int tok0) {
@@ -128,68 +130,160 @@ __device__ __forceinline__ int pf_steps_of_rank(int group, int P, int C, int n_t
 // first KV tile of piece i when nk steps are cut into k pieces
 __device__ __forceinline__ int pf_piece_begin(int nk, int k, int i) { return (int)(((long long)nk * i) / k); }
 
-template <bool kMulti>
-__device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p) {
-    PfPlan plan;
+// k ~ sqrt(steps / 6): a piece costs its steps plus a merge that grows with k (about six steps' worth per piece
+// merged); never pieces shorter than the minimum.
+__device__ __forceinline__ int pf_pieces_for(int steps) {
+    int k = 1;
+    while ((k + 1) * (k + 1) * 6 <= steps) ++k;
+    return max(1, min(k, steps / kPfMinPieceSteps));
+}
+
+// Several chunks in one iteration: the tail items (the last n_items mod gridDim ones) belong to chunks of very
+// different lengths, e.g. the end of a long prompt next to the start of a new one.  Each chunk gets its own piece
+// count, sized by its shortest item; while the tail entries outnumber the CTAs, the chunk with the shortest pieces
+// gives one up.  Run by one whole warp in the kernel prologue, lane j owning chunk j; fills the chunk table:
+// fields 0-3 the descriptors, 4 pieces per tail item, 5 items before the chunk, 6 tail entries before the chunk's
+// tail items (fields 5 and 6 hold INT_MAX where nothing may match), then the plan's totals.
+__device__ __forceinline__ void pf_fill_chunk_table(const MixedParams& p, int* tbl) {
+    const int lane = threadIdx.x & 31;
     const int G = (int)gridDim.x;
-    plan.n_items = 0;
+    int P = 0, C = 0, row0 = 0, page0 = 0;
+#pragma unroll
+    for (int j = 0; j < kMaxChunks; ++j)
+        if (lane == j) {
+            P = p.cP[j];
+            C = p.cC[j];
+            row0 = p.cRow0[j];
+            page0 = p.cPage0[j];
+        }
+    const bool live = lane < p.nchunks;
+    const int n_tp = live ? pf_num_groups(p.group, C) : 0;
+    const int cnt = n_tp * p.Hkv;
+    auto scan = [&](int v) {  // inclusive, over the first kMaxChunks lanes
+        for (int d = 1; d < kMaxChunks; d <<= 1) {
+            const int u = __shfl_up_sync(0xffffffffu, v, d);
+            if (lane >= d) v += u;
+        }
+        return v;
+    };
+    const int incl = scan(cnt);
+    const int before = incl - cnt;
+    const int n_items = __shfl_sync(0xffffffffu, incl, kMaxChunks - 1);
+    const int n_whole = n_items - n_items % G;
+    const int tail = max(0, before + cnt - max(before, n_whole));
+    int longest = 0, shortest = 0x7fffffff;
+    if (n_tp > 0) {
+        longest = pf_steps_of_rank(p.group, P, C, n_tp, 0);
+        shortest = pf_steps_of_rank(p.group, P, C, n_tp, n_tp - 1);
+    }
+    int k = tail > 0 ? pf_pieces_for(shortest) : 1;
+    int total = __reduce_add_sync(0xffffffffu, tail * k);
+    while (total > G) {  // warp-uniform
+        const int key = (tail > 0 && k > 1) ? (((shortest / k) << 5) | lane) : 0x7fffffff;
+        const int best = __reduce_min_sync(0xffffffffu, key);
+        if (best == 0x7fffffff) break;  // every k is 1: the tail holds fewer items than there are CTAs
+        if (key == best) k -= 1;
+        total -= __shfl_sync(0xffffffffu, tail, best & 31);
+    }
+    const int acc = scan(tail * k) - tail * k;
+    longest = __reduce_max_sync(0xffffffffu, longest);
+    shortest = __reduce_min_sync(0xffffffffu, shortest);
+    const int k0 = __shfl_sync(0xffffffffu, k, 0);
+    if (lane < kMaxChunks) {
+        tbl[lane] = P;
+        tbl[kMaxChunks + lane] = C;
+        tbl[2 * kMaxChunks + lane] = row0;
+        tbl[3 * kMaxChunks + lane] = page0;
+        tbl[4 * kMaxChunks + lane] = k;
+        tbl[5 * kMaxChunks + lane] = live ? before : 0x7fffffff;
+        tbl[6 * kMaxChunks + lane] = tail > 0 ? acc : 0x7fffffff;
+    }
+    if (lane == 0) {
+        int* tot = tbl + kChunkTotals;
+        tot[0] = n_items;
+        tot[1] = n_whole;
+        tot[2] = n_whole + total;
+        tot[3] = longest;
+        tot[4] = shortest;
+        tot[5] = n_whole == 0 ? k0 : 1;
+    }
+}
+
+template <bool kMulti>
+__device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p, uint32_t table) {
+    PfPlan plan;
+    plan.table = table;
+    if constexpr (kMulti) {  // worked out once per CTA by pf_fill_chunk_table
+        const uint32_t tot = table + kChunkTotals * 4;
+        plan.n_items = lds_s32(tot);
+        plan.n_whole = lds_s32(tot + 4);
+        plan.n_entries = lds_s32(tot + 8);
+        plan.longest = lds_s32(tot + 12);
+        plan.shortest = lds_s32(tot + 16);
+        plan.pieces = lds_s32(tot + 20);
+        return plan;
+    }
+    const int G = (int)gridDim.x;
+    const int n_tp = pf_num_groups(p.group, p.cC[0]);
+    plan.n_items = n_tp * p.Hkv;
     plan.longest = 0;
     plan.shortest = 0x7fffffff;
-#pragma unroll
-    for (int j = 0; j < kMaxChunks; ++j) {
-        if (j < (kMulti ? p.nchunks : 1)) {
-            const int n_tp = pf_num_groups(p.group, p.cC[j]);
-            plan.n_items += n_tp * p.Hkv;
-            if (n_tp > 0) {
-                plan.longest = max(plan.longest, pf_steps_of_rank(p.group, p.cP[j], p.cC[j], n_tp, 0));
-                plan.shortest = min(plan.shortest, pf_steps_of_rank(p.group, p.cP[j], p.cC[j], n_tp, n_tp - 1));
-            }
-        }
+    if (n_tp > 0) {
+        plan.longest = pf_steps_of_rank(p.group, p.cP[0], p.cC[0], n_tp, 0);
+        plan.shortest = pf_steps_of_rank(p.group, p.cP[0], p.cC[0], n_tp, n_tp - 1);
     }
     const int r = plan.n_items % G;
     plan.n_whole = plan.n_items - r;
     plan.pieces = 1;
-    if (r > 0) {
-        // the tail items are short ones; size the pieces by the shortest item
-        // A piece costs its steps plus a merge that grows with k (about six steps' worth per piece merged), so
-        // k ~ sqrt(steps / 6); never more pieces than fit side by side, never pieces shorter than the minimum.
-        const int shortest = plan.shortest;
-        int k = 1;
-        while ((k + 1) * (k + 1) * 6 <= shortest) ++k;
-        plan.pieces = max(1, min(min(G / r, k), shortest / kPfMinPieceSteps));
-    }
+    // the tail items are short ones; size the pieces by the shortest item, never more pieces than fit side by side
+    if (r > 0) plan.pieces = min(G / r, pf_pieces_for(plan.shortest));
     if (plan.pieces == 1) plan.n_whole = plan.n_items;
     plan.n_entries = plan.n_whole + (plan.n_items - plan.n_whole) * plan.pieces;
-    plan.prefix = nullptr;
     return plan;
 }
 
 template <bool kMulti>
 __device__ __forceinline__ PfItem pf_entry(const MixedParams& p, const PfPlan& plan, int entry) {
     PfItem it;
-    if (entry < plan.n_whole) {
-        it.item = entry;
-        it.piece = 0;
-    } else {
-        it.item = plan.n_whole + (entry - plan.n_whole) / plan.pieces;
-        it.piece = (entry - plan.n_whole) % plan.pieces;
-    }
-    // the item's chunk: the last one whose items start at or before it.  The chunks' item counts are recomputed here
-    // (a table of them would sit in registers of every role for the whole phase); indices into the kernel parameters
-    // are compile-time constants so that the parameters stay in constant memory.
-    int before = 0, count = 0, cP = p.cP[0], cC = p.cC[0];
+    it.pieces = plan.pieces;
+    it.slot0 = 0;
     it.chunk = 0;
-#pragma unroll
-    for (int j = 0; j < kMaxChunks; ++j)
-        if (kMulti && j < p.nchunks) {
-            if (it.item >= count) {
-                before = count;
-                it.chunk = j;
-                cP = p.cP[j];
-                cC = p.cC[j];
-            }
-            count += pf_num_groups(p.group, p.cC[j]) * p.Hkv;
+    int before = 0, cP = p.cP[0], cC = p.cC[0];
+    if constexpr (!kMulti) {
+        if (entry < plan.n_whole) {
+            it.item = entry;
+            it.piece = 0;
+        } else {
+            it.item = plan.n_whole + (entry - plan.n_whole) / plan.pieces;
+            it.piece = (entry - plan.n_whole) % plan.pieces;
+            it.slot0 = (it.item - plan.n_whole) * plan.pieces;
         }
+    } else {
+        // The entry's chunk is the last one whose threshold it reaches: for a whole item the items before the chunk,
+        // for a tail entry the tail entries before the chunk's (tail entries are numbered chunk by chunk: a chunk's
+        // tail items times the chunk's own piece count; the first chunk that has tail items has threshold 0).
+        const bool whole = entry < plan.n_whole;
+        const int key = whole ? entry : entry - plan.n_whole;
+        const uint32_t thr = plan.table + (whole ? 5 : 6) * kMaxChunks * 4;
+#pragma unroll
+        for (int j = 1; j < kMaxChunks; ++j)
+            if (key >= lds_s32(thr + j * 4)) it.chunk = j;
+        const uint32_t col = plan.table + it.chunk * 4;
+        cP = lds_s32(col);
+        cC = lds_s32(col + kMaxChunks * 4);
+        before = lds_s32(col + 5 * kMaxChunks * 4);
+        if (whole) {
+            it.item = entry;
+            it.piece = 0;
+        } else {
+            it.pieces = lds_s32(col + 4 * kMaxChunks * 4);
+            const int rel = key - lds_s32(col + 6 * kMaxChunks * 4);
+            const int idx = rel / it.pieces;
+            it.item = max(before, plan.n_whole) + idx;
+            it.piece = rel - idx * it.pieces;
+            it.slot0 = key - it.piece;
+        }
+    }
     const int local = it.item - before;
     const int rank = local / p.Hkv;
     it.kvh = local % p.Hkv;
@@ -203,11 +297,9 @@ __device__ __forceinline__ PfItem pf_entry(const MixedParams& p, const PfPlan& p
     if (entry < plan.n_whole) {
         it.j0 = 0;
         it.j1 = it.nk;
-        it.slot0 = 0;
     } else {
-        it.j0 = pf_piece_begin(it.nk, plan.pieces, it.piece);
-        it.j1 = pf_piece_begin(it.nk, plan.pieces, it.piece + 1);
-        it.slot0 = (it.item - plan.n_whole) * plan.pieces;
+        it.j0 = pf_piece_begin(it.nk, it.pieces, it.piece);
+        it.j1 = pf_piece_begin(it.nk, it.pieces, it.piece + 1);
     }
     return it;
 }
@@ -578,8 +670,8 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
     // ---- the item is shared with other CTAs: publish this piece, the last piece to arrive merges all of them ----
     // pieces of this item that hold steps of tile t: 0 .. last_piece (pieces are never empty: k <= nk / 4)
     int last_piece = 0;
-    for (int i = 1; i < plan.pieces; ++i)
-        if (pf_piece_begin(it.nk, plan.pieces, i) < it.nkv[t]) last_piece = i;
+    for (int i = 1; i < it.pieces; ++i)
+        if (pf_piece_begin(it.nk, it.pieces, i) < it.nkv[t]) last_piece = i;
     const int n_mine = last_piece + 1;
     const int my_slot = it.slot0 + it.piece;
     {

@@ -137,6 +137,7 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
     fallback_iters = fallback_run = 0
     fallbacks_since_table = reprofiles = 0
     prompts_per_chunk_iter = []
+    miss_samples = []        # the first few iterations that ran a chunk and overran the earliest deadline
     prefill_tokens = 0
     wall0 = time.time()
     while done < len(reqs):
@@ -262,6 +263,11 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
         if n and now > true_deadline:
             if c > 0:
                 misses_chunk += 1
+                if len(miss_samples) < 16:
+                    miss_samples.append({"n": n, "total_ctx": int(total_ctx), "chunks": [int(cj) for _, cj in admitted],
+                                         "prefixes": [int(r.prefilled) for r, _ in admitted], "budget_ns": budget,
+                                         "predicted_ns": int(predicted), "measured_ns": dt,
+                                         "late_ns": int(now - true_deadline)})
             else:
                 misses_decode_only += 1
         if flags & B.SW_F_DECODE_INFEASIBLE:
@@ -333,6 +339,7 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
         "fallback_iterations": fallback_iters, "reprofiles": reprofiles,
         "mean_prompts_per_chunk_iteration": float(np.mean(prompts_per_chunk_iter)) if prompts_per_chunk_iter else 0.0,
         "margin_ppm": margin_ppm, "c_max": c_max, "quantum": quantum, "wall_s": time.time() - wall0,
+        "miss_samples": miss_samples,
     }
 
 
@@ -355,6 +362,8 @@ def main(argv=None):
     ap.add_argument("--table", default=None, help="JSON cost table to reuse; measured first when absent")
     ap.add_argument("--table-reps", type=int, default=8)
     ap.add_argument("--max-prefills", type=int, default=1, help="prompts admitted per iteration (first fit when > 1)")
+    ap.add_argument("--telemetry", action="store_true",
+                    help="residual feedback (Sec. 3.3): add the P99 residual of the (n, L) bin to the controller's margin")
     ap.add_argument("--out", default="bursty_results.json")
     args = ap.parse_args(argv)
 
@@ -394,10 +403,14 @@ def main(argv=None):
         for tpot in args.tpot_ms:
             for policy in args.policies:
                 log(f"run: rate x{scale} tpot={tpot} ms policy={policy}")
+                tele = B.Telemetry([1, 4, 16, 48, 128, 256], [0, 64, 256, 1024, 2048, 4096]) if args.telemetry else None
                 res = run_trace(scaled, tpot, table, execute, shape, args.pages, policy=policy, c_max=args.c_max,
                                 margin_ppm=args.margin_ppm, max_decode=max_decode, ctx_cap=tab["ctx_grid"][-1], log=log,
-                                max_prefills=args.max_prefills, prefix_cap=tab["prefix_grid"][-1])
+                                max_prefills=args.max_prefills, prefix_cap=tab["prefix_grid"][-1], telemetry=tele)
                 B.sw_check_status(ctx)
+                if tele is not None:
+                    res["telemetry"] = tele.totals()
+                    tele.close()
                 res["rate_scale"] = scale
                 log(json.dumps(res))
                 results["runs"].append(res)

@@ -51,6 +51,11 @@ CASES = {
     "prefill_only_eight": (W.TINY, 600, [], [(0, 40), (16, 16), (100, 257), (3, 5), (640, 64), (0, 1), (31, 33), (200, 100)]),
     "group8": (W.AttnShape(8, 1, 128), 300, [40, 500], [(64, 200), (300, 17)]),
     "llama_mixed": (W.LLAMA, 1200, [900, 2000, 333, 1500, 16], [(2048, 700), (0, 300), (512, 512)]),
+    # chunks whose items are cut into different numbers of KV pieces: the end of a long prompt beside a new prompt,
+    # three different counts, and counts trimmed because the pieces would outnumber the CTAs
+    "long_end_new_start": (W.AttnShape(8, 2, 128), 400, [17, 300], [(3400, 70), (0, 50)]),
+    "three_piece_counts": (W.AttnShape(8, 2, 128), 900, [64], [(8000, 100), (3300, 64), (0, 30)]),
+    "pieces_trimmed_to_grid": (W.AttnShape(16, 16, 64), 1000, [100], [(9000, 300), (4000, 500)]),
 }
 
 
