@@ -199,33 +199,37 @@ def sweep_multichunk(reps: int, log) -> list:
     dev = torch.device("cuda", 0)
     shape = W.LLAMA
     rows = []
-    for total, prefix in ((512, 512), (2048, 4096)):
+    equal = [[(prefix, total // k)] * k for total, prefix in ((512, 512), (2048, 4096)) for k in (1, 2, 4, 8)]
+    # chunks of very different lengths: the end of a long prompt beside the start of new ones, and the same tokens as
+    # one chunk of the long prompt for comparison
+    unequal = [[(28672, 512)], [(28672, 256), (0, 256)], [(28672, 128), (4096, 128), (0, 256)]]
+    for chunks in equal + unequal:
         for n in (0, 64):
-            for k in (1, 2, 4, 8):
-                rng = W.rng_for(1)
-                lens = rng.integers(256, 2048, size=n, endpoint=True) if n else []
-                chunks = [(prefix, total // k)] * k
-                need = sum(-(-int(x) // 16) for x in lens) + k * (-(-(prefix + total // k) // 16)) + 64
-                batch = W.make_multi_batch(shape, need, lens, chunks, rng)
-                pools = []
-                for layer in range(4):
-                    t = torch.empty(batch.num_pages * shape.page_elems, dtype=torch.bfloat16, device=dev)
-                    W.fill_normal_bf16_(t, W.SEED_BASE + 700 + layer)
-                    pools.append(t)
-                pages = int(batch.prefill_pages.shape[0] + batch.decode_pages.shape[0])
-                ctx = B.Context(shape, batch.num_pages, batch.chunk_len, max(n, 1), pages + 16)
-                q = torch.randn(batch.num_rows, shape.num_q_heads, shape.head_dim, device=dev).to(torch.bfloat16)
-                out = torch.empty_like(q)
-                p50, p99, _ = B.sw_cost_probe(ctx, pools, B.DeviceBatch(batch, dev), q, out, warmup=2, reps=reps)
-                B.sw_check_status(ctx)
-                flops = 4 * shape.num_q_heads * shape.head_dim * k * ((total // k) * prefix + (total // k) * (total // k + 1) // 2)
-                row = {"prefill_tokens": total, "prefix_of_each": prefix, "chunks": k, "decodes": n, "us_p50": p50 / 4e3,
-                       "us_p99": p99 / 4e3, "prefill_gflop": flops / 1e9}
-                rows.append(row)
-                log(f"tokens {total:5d} in {k} chunk(s) at prefix {prefix:5d}, {n:3d} decodes: {row['us_p50']:8.1f} us "
-                    f"(p99 {row['us_p99']:.1f}), {flops / 1e9:.1f} GFLOP of prefill")
-                del ctx, pools
-                torch.cuda.empty_cache()
+            rng = W.rng_for(1)
+            lens = rng.integers(256, 2048, size=n, endpoint=True) if n else []
+            k, total, prefix = len(chunks), sum(c for _, c in chunks), chunks[0][0]
+            need = sum(-(-int(x) // 16) for x in lens) + sum(-(-(P + C) // 16) for P, C in chunks) + 64
+            batch = W.make_multi_batch(shape, need, lens, chunks, rng)
+            pools = []
+            for layer in range(4):
+                t = torch.empty(batch.num_pages * shape.page_elems, dtype=torch.bfloat16, device=dev)
+                W.fill_normal_bf16_(t, W.SEED_BASE + 700 + layer)
+                pools.append(t)
+            pages = int(batch.prefill_pages.shape[0] + batch.decode_pages.shape[0])
+            ctx = B.Context(shape, batch.num_pages, batch.chunk_len, max(n, 1), pages + 16)
+            q = torch.randn(batch.num_rows, shape.num_q_heads, shape.head_dim, device=dev).to(torch.bfloat16)
+            out = torch.empty_like(q)
+            p50, p99, _ = B.sw_cost_probe(ctx, pools, B.DeviceBatch(batch, dev), q, out, warmup=2, reps=reps)
+            B.sw_check_status(ctx)
+            flops = 4 * shape.num_q_heads * shape.head_dim * sum(C * P + C * (C + 1) // 2 for P, C in chunks)
+            row = {"prefill_tokens": total, "prefix_of_each": prefix, "chunks": k, "decodes": n, "us_p50": p50 / 4e3,
+                   "chunk_list": [list(c) for c in chunks],
+                   "us_p99": p99 / 4e3, "prefill_gflop": flops / 1e9}
+            rows.append(row)
+            log(f"tokens {total:5d} in {k} chunk(s) {chunks if len(set(chunks)) > 1 else 'at prefix ' + str(prefix)}, {n:3d} decodes: {row['us_p50']:8.1f} us "
+                f"(p99 {row['us_p99']:.1f}), {flops / 1e9:.1f} GFLOP of prefill")
+            del ctx, pools
+            torch.cuda.empty_cache()
     return rows
 
 
