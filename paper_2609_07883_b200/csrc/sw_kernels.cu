@@ -160,6 +160,10 @@ struct Geo {
     static constexpr int kSmemBytes = kMiscOffset + 768;   // 64 ints scan scratch and flags, the plan's counters, the chunk table
 };
 
+#ifndef SW_WIDE_MERGE_SPLITS
+#define SW_WIDE_MERGE_SPLITS 24
+#endif
+constexpr int kWideMergeSplits = SW_WIDE_MERGE_SPLITS;  // from this many splits of a request on, g units share the merge
 constexpr int kOneRoundMaxPages = 48;  // longest unit (pages) for which one round of units is planned
 constexpr int kPlanCounters = 8;       // shared counters of the plan's block sums, zeroed in the kernel prologue
 // When the CTAs of a single wave of prefill entries turn to decode units: a fixed start-up plus a time per 128-key
@@ -376,10 +380,11 @@ __device__ __forceinline__ void issue_page(const CUtensorMap* kvp_map, const War
 // Merge of the splits of one (request, kv head) by the last unit to arrive, all rows together so that the loads of
 // one pass are in flight at once.  G >= group size is a compile-time bound: rows beyond the group read row 0 with
 // weight zero, which keeps the loops free of branches.  Slots of the splits are Hkv apart.
-template <int D, int G>
-__device__ __forceinline__ void merge_splits(const MixedParams& p, const Unit& u) {
+// The warp merges rows [row0, row0 + nrows) of the group (all of them, or one row when several units share the merge);
+// J = splits whose partial outputs are loaded together.
+template <int D, int G, int J = (G >= 8 ? 2 : (G == 4 ? 4 : 8))>
+__device__ __forceinline__ void merge_splits(const MixedParams& p, const Unit& u, int row0, int nrows) {
     constexpr int V = D / 32;                 // output columns per lane
-    constexpr int J = G >= 8 ? 2 : (G == 4 ? 4 : 8);  // splits whose partial outputs are loaded together
     const int lane = threadIdx.x & 31;
     const int g = p.group;
     const int slot0 = u.slot - u.split * p.Hkv;
@@ -400,7 +405,7 @@ __device__ __forceinline__ void merge_splits(const MixedParams& p, const Unit& u
         float ms[G], ls[G];
 #pragma unroll
         for (int r = 0; r < G; ++r) {
-            const int rr = r < g ? r : 0;
+            const int rr = row0 + (r < nrows ? r : 0);
             ms[r] = __ldcg(ml0 + sidx * ml_stride + rr);
             ls[r] = __ldcg(ml0 + sidx * ml_stride + kMaxGroup + rr);
         }
@@ -440,10 +445,10 @@ __device__ __forceinline__ void merge_splits(const MixedParams& p, const Unit& u
         for (int r = 0; r < G; ++r) {
             float ms = m_first[r];
             if (s0 > 0) {
-                ms = __ldcg(ml0 + min(s0 + lane, ns - 1) * ml_stride + (r < g ? r : 0));
+                ms = __ldcg(ml0 + min(s0 + lane, ns - 1) * ml_stride + row0 + (r < nrows ? r : 0));
                 if (s0 + lane >= ns) ms = -INFINITY;
             }
-            w[r] = (ms == -INFINITY || r >= g) ? 0.f : fast_exp2((ms - m_all[r]) * p.sm_scale_log2);
+            w[r] = (ms == -INFINITY || r >= nrows) ? 0.f : fast_exp2((ms - m_all[r]) * p.sm_scale_log2);
         }
         const int cnt = min(32, ns - s0);
         for (int j0 = 0; j0 < cnt; j0 += J) {
@@ -453,7 +458,7 @@ __device__ __forceinline__ void merge_splits(const MixedParams& p, const Unit& u
                 const float* src = po0 + (s0 + min(j0 + j, cnt - 1)) * po_stride;
 #pragma unroll
                 for (int r = 0; r < G; ++r) {
-                    const float* row = src + (r < g ? r : 0) * D;
+                    const float* row = src + (row0 + (r < nrows ? r : 0)) * D;
                     if constexpr (V == 4) {
                         const float4 t = __ldcg(reinterpret_cast<const float4*>(row));
                         x[j][r][0] = t.x, x[j][r][1] = t.y, x[j][r][2] = t.z, x[j][r][3] = t.w;
@@ -477,9 +482,9 @@ __device__ __forceinline__ void merge_splits(const MixedParams& p, const Unit& u
     }
 #pragma unroll
     for (int r = 0; r < G; ++r) {
-        if (r < g) {
+        if (r < nrows) {
             const float inv = 1.f / l_all[r];
-            const int hd = u.kvh * g + r;
+            const int hd = u.kvh * g + row0 + r;
             __nv_bfloat16* dst = p.out + ((int64_t)u.q_row * p.Hq + hd) * D + lane * V;
             if constexpr (V == 4) {
                 *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16x2(acc[r][0] * inv, acc[r][1] * inv),
@@ -702,7 +707,40 @@ __device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const
             p.part_ml[(int64_t)u.slot * (2 * kMaxGroup) + kMaxGroup + qrow_in_group] = l_run;
         }
     }
-    const bool merger = __shfl_sync(0xffffffffu, ticket, 0) == u.nsplit - 1;
+    ticket = __shfl_sync(0xffffffffu, ticket, 0);
+    if (g > 1 && u.nsplit >= kWideMergeSplits) {
+        // Many splits (one long context cut for all the warps): a single warp would load their partial outputs a few
+        // at a time.  The units that drew the last g tickets share the merge, one row of the group each; every unit,
+        // those included, publishes its partial result, and the last merger to finish re-arms the counters.
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) atomicAdd(&p.ready[u.ticket], 1);
+        const int row = ticket - (u.nsplit - g);
+        if (row < 0) return true;
+        int ok = 1;
+        if (lane == 0) {
+            const long long t0 = clock64();
+            while (ld_acquire_gpu(&p.ready[u.ticket]) < u.nsplit) {
+                if (clock64() - t0 > kWaitBudgetCycles) {
+                    ok = 0;
+                    break;
+                }
+                __nanosleep(64);
+            }
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) {
+            if (lane == 0) report(p.ctrl, SW_ERR_DEVICE_TIMEOUT, kSiteWait, u.q_row);
+            return false;
+        }
+        merge_splits<D, 1, 16>(p, u, row, 1);
+        if (lane == 0 && atomicAdd(&p.ready[u.ticket], 1) == u.nsplit + g - 1) {
+            p.tickets[u.ticket] = 0;  // ready for the next launch
+            p.ready[u.ticket] = 0;
+        }
+        return true;
+    }
+    const bool merger = ticket == u.nsplit - 1;
     if (!merger) {
         __threadfence();
         __syncwarp();
@@ -730,10 +768,10 @@ __device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const
         return false;
     }
     switch (g) {
-        case 1: merge_splits<D, 1>(p, u); break;
-        case 2: merge_splits<D, 2>(p, u); break;
-        case 4: merge_splits<D, 4>(p, u); break;
-        default: merge_splits<D, kMaxGroup>(p, u); break;
+        case 1: merge_splits<D, 1>(p, u, 0, 1); break;
+        case 2: merge_splits<D, 2>(p, u, 0, 2); break;
+        case 4: merge_splits<D, 4>(p, u, 0, 4); break;
+        default: merge_splits<D, kMaxGroup>(p, u, 0, g); break;
     }
     return true;
 }

@@ -362,6 +362,8 @@ def main(argv=None):
     ap.add_argument("--table", default=None, help="JSON cost table to reuse; measured first when absent")
     ap.add_argument("--table-reps", type=int, default=8)
     ap.add_argument("--max-prefills", type=int, default=1, help="prompts admitted per iteration (first fit when > 1)")
+    ap.add_argument("--ttft-slo-ms", type=float, default=None,
+                    help="also count the requests that meet both SLOs and the goodput (Sec. 4.3)")
     ap.add_argument("--telemetry", action="store_true",
                     help="residual feedback (Sec. 3.3): add the P99 residual of the (n, L) bin to the controller's margin")
     ap.add_argument("--out", default="bursty_results.json")
@@ -406,7 +408,8 @@ def main(argv=None):
                 tele = B.Telemetry([1, 4, 16, 48, 128, 256], [0, 64, 256, 1024, 2048, 4096]) if args.telemetry else None
                 res = run_trace(scaled, tpot, table, execute, shape, args.pages, policy=policy, c_max=args.c_max,
                                 margin_ppm=args.margin_ppm, max_decode=max_decode, ctx_cap=tab["ctx_grid"][-1], log=log,
-                                max_prefills=args.max_prefills, prefix_cap=tab["prefix_grid"][-1], telemetry=tele)
+                                max_prefills=args.max_prefills if policy == "sloweave" else 1, prefix_cap=tab["prefix_grid"][-1],
+                                telemetry=tele, ttft_slo_ms=args.ttft_slo_ms)
                 B.sw_check_status(ctx)
                 if tele is not None:
                     res["telemetry"] = tele.totals()

@@ -331,3 +331,25 @@ def test_a_wait_that_cannot_succeed_gives_up_and_the_context_stays_usable(gpu, o
     assert code == r.B.SW_ERR_DEVICE_TIMEOUT and (detail & 0xFFFFFF) == 0xABCD
     assert r.status() == (0, 0)
     run_and_compare(gpu, oracle, batch, t, what="after a timed-out wait")
+
+
+@pytest.mark.parametrize("heads", [(8, 1, 128), (8, 2, 128), (4, 2, 64), (8, 8, 64)])
+def test_many_splits_of_one_request_share_the_merge(gpu, oracle, heads):
+    """One long context beside a short one is cut into dozens of units per KV head; from a few dozen splits on, the
+    units that draw the last tickets merge one row of the group each (group sizes 8, 4, 2; group 1 keeps the single
+    merger).  Run twice: the shared counters must re-arm themselves."""
+    rng = np.random.default_rng(35)
+    lens = [20011, 500]
+    need = sum(-(-x // 16) for x in lens)
+    batch = W.make_batch(W.AttnShape(*heads), need + 8, lens, 0, 0, rng)
+    t = W.host_tensors(batch, rng)
+    run_and_compare(gpu, oracle, batch, t, what=f"wide merge {heads}")
+    r = gpu.Runner(batch, t)
+    r.append()
+    r.attend()
+    first, _ = r.results()
+    r.out.zero_()
+    r.attend()
+    second, _ = r.results()
+    assert r.status() == (0, 0)
+    assert np.array_equal(first, second)
