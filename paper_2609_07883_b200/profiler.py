@@ -233,6 +233,39 @@ def sweep_multichunk(reps: int, log) -> list:
     return rows
 
 
+def sweep_few_long_contexts(reps: int, log) -> list:
+    """Decode-only launches over one or four long contexts: every warp streams a slice of the same request, and the
+    slices of a (request, KV head) are merged by the units that finish last."""
+    import torch
+
+    from . import binding as B
+
+    dev = torch.device("cuda", 0)
+    shape = W.LLAMA
+    rows = []
+    for lens in ([8192], [65536], [196608], [600000], [16384] * 4, [49152] * 4):
+        need = sum(-(-x // shape.page_size) for x in lens) + 64
+        batch = W.make_batch(shape, need, lens, 0, 0, W.rng_for(2))
+        pools = []
+        for layer in range(2):
+            t = torch.empty(batch.num_pages * shape.page_elems, dtype=torch.bfloat16, device=dev)
+            W.fill_normal_bf16_(t, W.SEED_BASE + 800 + layer)
+            pools.append(t)
+        ctx = B.Context(shape, batch.num_pages, 1, len(lens), int(batch.decode_pages.shape[0]) + 16)
+        q = torch.randn(batch.num_rows, shape.num_q_heads, shape.head_dim, device=dev).to(torch.bfloat16)
+        out = torch.empty_like(q)
+        p50, p99, _ = B.sw_cost_probe(ctx, pools, B.DeviceBatch(batch, dev), q, out, warmup=3, reps=reps)
+        B.sw_check_status(ctx)
+        kv_bytes = sum(lens) * 2 * shape.num_kv_heads * shape.head_dim * 2
+        row = {"contexts": lens, "us_p50": p50 / 2e3, "us_p99": p99 / 2e3, "kv_bytes": kv_bytes,
+               "gbs": kv_bytes / (p50 / 2e9) / 1e9}
+        rows.append(row)
+        log(f"contexts {lens}: {row['us_p50']:8.1f} us (p99 {row['us_p99']:.1f}), {kv_bytes / 1e6:.0f} MB of K/V, {row['gbs']:.0f} GB/s")
+        del ctx, pools
+        torch.cuda.empty_cache()
+    return rows
+
+
 def main(argv=None):
     import argparse
     import sys
@@ -240,13 +273,15 @@ def main(argv=None):
     from . import build
 
     ap = argparse.ArgumentParser(description="cost surface of a named workload: mixed / prefill-only / decode-only launches")
-    ap.add_argument("--config", choices=["chat", "mixed", "long", "multichunk"], default="mixed")
+    ap.add_argument("--config", choices=["chat", "mixed", "long", "multichunk", "longcontext"], default="mixed")
     ap.add_argument("--reps", type=int, default=10)
     ap.add_argument("--out", default=None)
     args = ap.parse_args(argv)
     build.build()
     if args.config == "multichunk":
         rows = sweep_multichunk(args.reps, lambda s: print(s, flush=True))
+    elif args.config == "longcontext":
+        rows = sweep_few_long_contexts(max(args.reps, 20), lambda s: print(s, flush=True))
     else:
         rows = sweep(args.config, args.reps, lambda s: print(s, flush=True))
     out = args.out or f"cost_surface_{args.config}.json"
