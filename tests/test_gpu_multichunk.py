@@ -148,3 +148,26 @@ def test_large_chunks_with_tail_pieces_sampled_rows(gpu, oracle):
         g = out[row0 + pairs[:, 0], pairs[:, 1]]
         gl = lse[row0 + pairs[:, 0], pairs[:, 1]]
         gpu.compare(g, gl, ref, ref_lse, f"tail pieces, rows from {row0}")
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3, 4])
+def test_random_mixes_of_long_and_short_chunks(gpu, oracle, seed):
+    """Two to eight chunks whose prefixes range from nothing to thousands of tokens: the chunks' items get different
+    numbers of KV pieces (or none), in every order of long and short chunks, beside a few decodes."""
+    rng = np.random.default_rng(700 + seed)
+    shape = [W.AttnShape(8, 2, 128), W.AttnShape(4, 4, 64), W.AttnShape(8, 1, 128), W.AttnShape(16, 4, 64)][seed - 1]
+    k = int(rng.integers(2, 9))
+    chunks = [(int(rng.choice([0, 0, 700, 3500, 9000])) + int(rng.integers(0, 40)), int(rng.integers(1, 200)))
+              for _ in range(k)]
+    lens = [int(x) for x in rng.integers(1, 3000, size=int(rng.integers(0, 5)))]
+    pages = sum(-(-(P + C) // 16) for P, C in chunks) + sum(-(-x // 16) for x in lens) + 16
+    batch = W.make_multi_batch(shape, pages, lens, chunks, rng, name=f"random mix {seed}")
+    t = W.host_tensors(batch, rng)
+    r = gpu.Runner(batch, t)
+    r.iterate()
+    out, lse = r.results()
+    assert r.status() == (0, 0)
+    pool, ref, ref_lse = oracle_rows(oracle, batch, t)
+    assert np.array_equal(gpu.torch_to_bits(r.pool), pool), "pool differs after append"
+    gpu.compare(out.reshape(-1, shape.head_dim), lse.reshape(-1), ref.reshape(-1, shape.head_dim), ref_lse.reshape(-1),
+                f"random mix {seed}: {chunks}")
