@@ -63,7 +63,7 @@ struct MixedParams {
     int target_items;   // split-KV units aimed at (<= max_items - n*Hkv)
     // scratch of prefill items finished by several CTAs
     float* pf_ml;        // [kMaxCtas][2][2][128]
-    float* pf_o;         // [kMaxCtas][2][128][D]
+    float* pf_o;         // [kMaxCtas][2][D / 4][128][4]
     int32_t* pf_tickets; // [items][2]
 };
 

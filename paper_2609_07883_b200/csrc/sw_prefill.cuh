@@ -89,6 +89,10 @@ __device__ __forceinline__ bool pf_wait(const PfShared& sh, int bar, uint32_t pa
 #define SW_PF_MIN_PIECE_STEPS 4
 #endif
 constexpr int kPfMinPieceSteps = SW_PF_MIN_PIECE_STEPS;
+#ifndef SW_PF_PIECE_COST
+#define SW_PF_PIECE_COST 1
+#endif
+constexpr int kPfPieceCost = SW_PF_PIECE_COST;  // steps' worth of work that cutting an item into one more piece costs
 
 struct PfPlan {
     int longest, shortest;             // steps of the longest and of the shortest item (items are numbered chunk by chunk)
@@ -130,11 +134,12 @@ __device__ __forceinline__ int pf_steps_of_rank(int group, int P, int C, int n_t
 // first KV tile of piece i when nk steps are cut into k pieces
 __device__ __forceinline__ int pf_piece_begin(int nk, int k, int i) { return (int)(((long long)nk * i) / k); }
 
-// k ~ sqrt(steps / 6): a piece costs its steps plus a merge that grows with k (about six steps' worth per piece
-// merged); never pieces shorter than the minimum.
+// k ~ sqrt(steps / cost): a piece costs its steps plus a merge that grows with k (about one step's worth per piece
+// merged, with partial results laid out so that publishing and merging are coalesced); never pieces shorter than the
+// minimum.
 __device__ __forceinline__ int pf_pieces_for(int steps) {
     int k = 1;
-    while ((k + 1) * (k + 1) * 6 <= steps) ++k;
+    while ((k + 1) * (k + 1) * kPfPieceCost <= steps) ++k;
     return max(1, min(k, steps / kPfMinPieceSteps));
 }
 
@@ -517,7 +522,7 @@ struct PfSoftmaxState {
 // per slot and tile: m[128], l[128] and O[128][D], all fp32.
 struct PfScratch {
     float* ml;         // [slots][2 tiles][2][128]
-    float* o;          // [slots][2 tiles][128][D]
+    float* o;          // [slots][2 tiles][D / 4 column chunks][128 rows][4]
     int32_t* tickets;  // [items][2 tiles]
     volatile int* flags;  // shared memory, one int per tile: ticket value seen by the warpgroup's thread 0
 };
@@ -676,20 +681,26 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
     const int my_slot = it.slot0 + it.piece;
     {
         float* ml = scr.ml + ((int64_t)my_slot * 2 + t) * 256;
-        float* po = scr.o + (((int64_t)my_slot * 2 + t) * 128 + row) * D;
+        // O of a (slot, tile) is stored by 16-byte column chunks: chunk q of all 128 rows, then chunk q + 1, so that
+        // the 32 rows of a warp write (and the merging warp reads) 512 contiguous bytes per instruction
+        float* po = scr.o + ((int64_t)my_slot * 2 + t) * 128 * D + row * 4;
         ml[row] = m_ref;
         ml[128 + row] = l_sum;
+#ifndef SW_EXP_NO_PUBLISH
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
             tmem_ld_32x32b_x32(o_addr + c * 32, v);
             tc_wait_ld();
 #pragma unroll
             for (int i = 0; i < 8; ++i)
-                *reinterpret_cast<uint4*>(po + c * 32 + i * 4) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                *reinterpret_cast<uint4*>(po + (c * 8 + i) * 512) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
         }
+#endif
     }
     tc_fence_before_sync();
+#ifndef SW_EXP_NO_FENCE
     __threadfence();
+#endif
     named_barrier_sync(2 + t, 128);
     if ((warp & 3) == 0 && lane == 0) scr.flags[t] = atomicAdd(&scr.tickets[it.item * 2 + t], 1);
     named_barrier_sync(2 + t, 128);
@@ -698,6 +709,9 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
     if (!merger) return true;
     __threadfence();
     if ((warp & 3) == 0 && lane == 0) scr.tickets[it.item * 2 + t] = 0;  // re-armed for the next launch
+#ifdef SW_EXP_NO_MERGE
+    return true;
+#endif
     const float* ml0 = scr.ml + ((int64_t)it.slot0 * 2 + t) * 256 + row;  // piece i: + i * 512 floats
     float m_all = -INFINITY;
 #pragma unroll 4
@@ -711,7 +725,7 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
     }
     const float inv = 1.f / l_all;
     // 64 output columns at a time keeps the accumulators small, so that the loads of two pieces are in flight
-    const float* o0 = scr.o + (((int64_t)it.slot0 * 2 + t) * 128 + row) * D;  // piece i: + i * 2 * 128 * D floats
+    const float* o0 = scr.o + ((int64_t)it.slot0 * 2 + t) * 128 * D + row * 4;  // piece i: + i * 2 * 128 * D floats
 #pragma unroll 1
     for (int c = 0; c < D / 64; ++c) {
         float acc[64];
@@ -721,10 +735,10 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
         for (int i = 0; i <= last_piece; ++i) {
             const float ms = __ldcg(ml0 + (int64_t)i * 512);
             const float w = ms == -INFINITY ? 0.f : fast_exp2(ms - m_all);
-            const float4* po = reinterpret_cast<const float4*>(o0 + (int64_t)i * 2 * 128 * D + c * 64);
+            const float* po = o0 + (int64_t)i * 2 * 128 * D + c * 16 * 512;
             float4 x[16];
 #pragma unroll
-            for (int q = 0; q < 16; ++q) x[q] = __ldcg(po + q);
+            for (int q = 0; q < 16; ++q) x[q] = __ldcg(reinterpret_cast<const float4*>(po + q * 512));
 #pragma unroll
             for (int q = 0; q < 16; ++q) {
                 acc[4 * q + 0] = fmaf(w, x[q].x, acc[4 * q + 0]);
