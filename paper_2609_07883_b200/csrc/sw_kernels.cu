@@ -163,7 +163,7 @@ struct Geo {
 #ifndef SW_WIDE_MERGE_SPLITS
 #define SW_WIDE_MERGE_SPLITS 24
 #endif
-constexpr int kWideMergeSplits = SW_WIDE_MERGE_SPLITS;  // from this many splits of a request on, g units share the merge
+constexpr int kWideMergeSplits = SW_WIDE_MERGE_SPLITS;  // from this many units of a request on, its last g units share the merge
 constexpr int kOneRoundMaxPages = 48;  // longest unit (pages) for which one round of units is planned
 constexpr int kPlanCounters = 8;       // shared counters of the plan's block sums, zeroed in the kernel prologue
 // When the CTAs of a single wave of prefill entries turn to decode units: a fixed start-up plus a time per 128-key
@@ -497,6 +497,17 @@ __device__ __forceinline__ void merge_splits(const MixedParams& p, const Unit& u
     }
 }
 
+// Which row of the group a unit of a request with many units merges (-1: none).  Not inlined: the rare case should
+// not cost the common one registers or instructions.
+__device__ __noinline__ int wide_merge_row(int nsplit, int split, int kvh, int g, int Hkv) {
+    const int d = nsplit - 1 - split;
+    if (nsplit >= 2 * g * Hkv) {
+        const int q = d >> 1;
+        return (!(d & 1) && q % Hkv == kvh && q / Hkv < g) ? q / Hkv : -1;
+    }
+    return d < g ? d : -1;
+}
+
 // Runs one unit; returns false if a bounded wait expired.
 template <int D>
 __device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const Unit& u, WarpRing<D>& ring, int fixed_items, bool pulls,
@@ -565,14 +576,21 @@ __device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const
     // round trip hides behind the last pages, and no warp hoards a unit while others are still idle.
     // With the claim the unit draws its ticket among the units of its (request, kv head): the last ticket makes it
     // the one that merges.  Both answers are read at the end of the unit, when they have long arrived.
-    bool claimed = false;
+    // A request cut into many units (kWideMergeSplits or more) has g mergers per kv head, fixed in advance among its
+    // last units, one query-head row each.  Such a unit will wait for the request's other units, so it must not hold
+    // a claimed unit meanwhile (another merger could be waiting for that one): it claims its next unit after the merge.
+    // With enough units the mergers of the different heads and rows are every other unit from the end (row j of head
+    // h: unit nsplit - 1 - 2 (j Hkv + h)), which puts them on different SMs; otherwise the last g units of each head.
+    const bool wide = g > 1 && u.nsplit >= kWideMergeSplits;
+    const int merge_row = wide ? wide_merge_row(u.nsplit, u.split, u.kvh, g, p.Hkv) : -1;
+    bool claimed = merge_row >= 0;
     int ticket = 0;  // lane 0
     auto claim_next = [&]() {
         if (!claimed && issued >= npg) {
             claimed = true;
             if (lane == 0) {
                 next_item = pulls ? fixed_items + atomicAdd(&p.ctrl[kCtrWork], 1) : 0x7fffffff;
-                if (u.nsplit > 1) ticket = atomicAdd(&p.tickets[u.ticket], 1);
+                if (u.nsplit > 1 && !wide) ticket = atomicAdd(&p.tickets[u.ticket], 1);
             }
         }
     };
@@ -707,16 +725,17 @@ __device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const
             p.part_ml[(int64_t)u.slot * (2 * kMaxGroup) + kMaxGroup + qrow_in_group] = l_run;
         }
     }
-    ticket = __shfl_sync(0xffffffffu, ticket, 0);
-    if (g > 1 && u.nsplit >= kWideMergeSplits) {
+    if (wide) {
         // Many splits (one long context cut for all the warps): a single warp would load their partial outputs a few
-        // at a time.  The units that drew the last g tickets share the merge, one row of the group each; every unit,
-        // those included, publishes its partial result, and the last merger to finish re-arms the counters.
+        // at a time.  Every unit publishes its partial result; g of the request's last units then merge one row of
+        // the group each.  A waiting merger holds no claimed unit, and the units it waits for are run by warps that wait
+        // for nothing or are claimed by such warps: a request has 24 units or more only if it holds 23 units' worth
+        // of pages, so at most target_items / 23 (request, kv head) pairs have mergers, fewer than 1500 warps even
+        // with groups of 8, and some warp is always free to claim.  The last merger to finish re-arms the counter.
         __threadfence();
         __syncwarp();
         if (lane == 0) atomicAdd(&p.ready[u.ticket], 1);
-        const int row = ticket - (u.nsplit - g);
-        if (row < 0) return true;
+        if (merge_row < 0) return true;
         int ok = 1;
         if (lane == 0) {
             const long long t0 = clock64();
@@ -733,13 +752,14 @@ __device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const
             if (lane == 0) report(p.ctrl, SW_ERR_DEVICE_TIMEOUT, kSiteWait, u.q_row);
             return false;
         }
-        merge_splits<D, 1, 16>(p, u, row, 1);
-        if (lane == 0 && atomicAdd(&p.ready[u.ticket], 1) == u.nsplit + g - 1) {
-            p.tickets[u.ticket] = 0;  // ready for the next launch
-            p.ready[u.ticket] = 0;
+        merge_splits<D, 1, 16>(p, u, merge_row, 1);
+        if (lane == 0) {
+            if (atomicAdd(&p.ready[u.ticket], 1) == u.nsplit + g - 1) p.ready[u.ticket] = 0;  // ready for the next launch
+            next_item = pulls ? fixed_items + atomicAdd(&p.ctrl[kCtrWork], 1) : 0x7fffffff;
         }
         return true;
     }
+    ticket = __shfl_sync(0xffffffffu, ticket, 0);
     const bool merger = ticket == u.nsplit - 1;
     if (!merger) {
         __threadfence();

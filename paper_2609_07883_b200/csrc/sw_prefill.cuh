@@ -686,7 +686,6 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
         float* po = scr.o + ((int64_t)my_slot * 2 + t) * 128 * D + row * 4;
         ml[row] = m_ref;
         ml[128 + row] = l_sum;
-#ifndef SW_EXP_NO_PUBLISH
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
             tmem_ld_32x32b_x32(o_addr + c * 32, v);
@@ -695,12 +694,9 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
             for (int i = 0; i < 8; ++i)
                 *reinterpret_cast<uint4*>(po + (c * 8 + i) * 512) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
         }
-#endif
     }
     tc_fence_before_sync();
-#ifndef SW_EXP_NO_FENCE
     __threadfence();
-#endif
     named_barrier_sync(2 + t, 128);
     if ((warp & 3) == 0 && lane == 0) scr.flags[t] = atomicAdd(&scr.tickets[it.item * 2 + t], 1);
     named_barrier_sync(2 + t, 128);
@@ -709,9 +705,6 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
     if (!merger) return true;
     __threadfence();
     if ((warp & 3) == 0 && lane == 0) scr.tickets[it.item * 2 + t] = 0;  // re-armed for the next launch
-#ifdef SW_EXP_NO_MERGE
-    return true;
-#endif
     const float* ml0 = scr.ml + ((int64_t)it.slot0 * 2 + t) * 256 + row;  // piece i: + i * 512 floats
     float m_all = -INFINITY;
 #pragma unroll 4
