@@ -353,3 +353,25 @@ def test_many_splits_of_one_request_share_the_merge(gpu, oracle, heads):
     second, _ = r.results()
     assert r.status() == (0, 0)
     assert np.array_equal(first, second)
+
+
+def test_many_long_requests_in_several_rounds(gpu, oracle):
+    """Six 30k-token requests over 8 KV heads: more pages than one round of units can take, so warps run several units
+    and pull them from the counter, and every request has dozens of units whose merge is shared by fixed mergers that
+    claim their next unit late.  Twice in a row: the counters must re-arm themselves."""
+    rng = np.random.default_rng(36)
+    shape = W.AttnShape(16, 8, 64)
+    lens = [30000 + 37 * i for i in range(6)]
+    need = sum(-(-x // 16) for x in lens)
+    batch = W.make_batch(shape, need + 8, lens, 0, 0, rng)
+    t = W.host_tensors(batch, rng)
+    run_and_compare(gpu, oracle, batch, t, what="several rounds of units, shared merges")
+    r = gpu.Runner(batch, t)
+    r.append()
+    r.attend()
+    first, _ = r.results()
+    r.out.zero_()
+    r.attend()
+    second, _ = r.results()
+    assert r.status() == (0, 0)
+    assert np.array_equal(first, second)
