@@ -175,6 +175,10 @@ constexpr int kPlanCounters = 8;       // shared counters of the plan's block su
 constexpr float kLateBaseUs = 1.0f, kLateStepUs = SW_LATE_STEP_US;
 constexpr float kDecodeBytesPerUs = 6.2e6f;
 constexpr int kMinEarlyCtas = 64;  // CTAs whose rings of page copies keep the memory system busy on their own
+#ifndef SW_MIN_LATE_CTAS
+#define SW_MIN_LATE_CTAS 24
+#endif
+constexpr int kMinLateCtas = SW_MIN_LATE_CTAS;  // fewer late CTAs than this: their delay is not worth units of two sizes
 struct Plan {
     const int* len;     // shared-memory copies of the context lengths and page-list offsets
     const int* indptr;
@@ -281,7 +285,7 @@ __device__ __forceinline__ Plan make_plan(const MixedParams& p, int* unit_prefix
         const float b_share = (float)total_pages - a_share;
         const float a_ragged = 0.6f * p.n * a_share / fmaxf(1.f, (float)total_pages);
         const float b_ragged = 0.6f * p.n - a_ragged;
-        if (G - late.ctas < kMinEarlyCtas || streamed < 0.25f * pages) {
+        if (G - late.ctas < kMinEarlyCtas || late.ctas < kMinLateCtas || streamed < 0.25f * pages) {
             // Too few early CTAs to keep the memory system busy on their own (the estimate of what they stream would
             // not hold), or a head start that is small next to the whole phase: one unit size, every warp pulls.
             split_a = split_b = plan_split_pages(p, total_pages, max(1, G * kWarps / p.Hkv));
