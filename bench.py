@@ -30,7 +30,7 @@ from paper_2609_07883_b200 import workloads as W  # noqa: E402
 # dram__bytes_read.sum + dram__bytes_write.sum of one sw_mixed_attn_kernel<128> launch of the default workload, from the
 # ncu capture summarised in profiles/sw_mixed_attn_kernel_chat_bench.md (298.8 MB read + 12.6 MB written; the launch
 # includes the fused KV append)
-NCU_TRAFFIC_DEFAULT_WORKLOAD = 310_712_064
+NCU_TRAFFIC_DEFAULT_WORKLOAD = 311_881_984
 NOMINAL_HBM_GBS = 8000.0
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
