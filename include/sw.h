@@ -15,6 +15,10 @@
  *     the caller's workspace).
  *   - `stream` is a cudaStream_t passed as void*.  Launching calls are asynchronous on that stream.
  *     One sw_ctx serves one stream at a time (its scratch and counters are shared by its launches).
+ *   - A context belongs to the device it was created on.  Launching calls (sw_kv_append, sw_mixed_attn_run,
+ *     sw_mixed_iteration_run, sw_mixed_iteration_host, the cost probes) require that device to be the caller's
+ *     current CUDA device and return SW_ERR_INVALID_ARG otherwise; no call changes the current device
+ *     (sw_create sets `device` for its own set-up and restores the caller's).
  *   - bf16 tensors are dense, row-major, innermost index last.
  *   - KV pool layout (elements, bf16):  [num_pages][2 (0 = K, 1 = V)][num_kv_heads][page_size][head_dim].
  *     The pool must hold finite values everywhere a page list can reach (initialise it with zeros): the
@@ -100,7 +104,9 @@ void sw_destroy(sw_ctx* ctx);
 /* KV manager step (Table 1): write this iteration's new K/V rows into the pool.  k_new / v_new are device
  * bf16 [C+n][num_kv_heads][head_dim].  Chunk row j goes to position P+j of the prompt's page list, decode row
  * i to position decode_kv_len[i]-1 of request i's list.  One kernel launch, asynchronous.  Page ids or
- * positions outside their list / the pool are skipped and reported by sw_check_status. */
+ * positions outside their list / the pool are skipped and reported by sw_check_status.  (The attention calls
+ * below report a page id outside the pool the same way and read page 0 in its place; their output for the
+ * affected rows is then meaningless.) */
 sw_status sw_kv_append(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const void* k_new, const void* v_new,
                        void* stream);
 
@@ -118,7 +124,10 @@ sw_status sw_mixed_attn_run(sw_ctx* ctx, const void* kv_pool, const sw_batch* ba
  * chunk's own keys and the decode units that reach a request's last page wait (bounded) until every CTA has done so.
  * Arguments as for the two calls.  Contract beyond theirs: no page of a decode request other than its last, and no
  * page below the chunk's first row, is written by this call (true of any page table in which requests own their
- * pages, shared prompt prefixes included).  Asynchronous. */
+ * pages, shared prompt prefixes included).  Asynchronous.
+ * The waits need every CTA of the persistent grid to be resident at once.  sw_create checks that (occupancy of the
+ * kernel times the SM count against the grid); on a device where it does not hold this call issues the append as a
+ * launch of its own before the attention launch, with the same results. */
 sw_status sw_mixed_iteration_run(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const void* k_new, const void* v_new,
                                  const void* q, void* out, float* lse, void* stream);
 
@@ -156,11 +165,14 @@ sw_status sw_cost_probe_iteration(sw_ctx* ctx, void* const* kv_pools, int32_t la
  * allocating library routine.
  * Limits: chunk_len must be 0, num_decode <= SW_STATIC_MAX_DECODE, num_kv_heads <= 8; anything larger is refused with
  * SW_ERR_WORKSPACE (SW_ERR_UNSUPPORTED for a prefill chunk).
+ * `device` must be the caller's current CUDA device (cudaSetDevice before the call); the call changes no device and
+ * refuses with SW_ERR_INVALID_ARG when another device is current.
  * The first call on a device looks up the array's device address, the device properties and the kernel attributes;
  * make that first call outside any stream capture.  All calls share the one array: it is cleared where it must start
  * at zero at the beginning of every call (on `stream`), so calls must not overlap on the GPU — issue them on one
  * stream, or order them yourself; overlapping calls race on the scratch.  Not thread-safe for concurrent first calls.
- * Asynchronous on `stream`; device-side problems are not reported by this variant (bad page ids are skipped). */
+ * Asynchronous on `stream`; device-side problems are not reported by this variant (a page id outside the pool is
+ * never fetched: page 0 is read in its place). */
 #define SW_STATIC_MAX_DECODE 128
 #define SW_STATIC_SCRATCH_BYTES (7u * 1024u * 1024u)
 sw_status sw_decode_attn_static(const sw_layout* layout, int device, const void* kv_pool, const sw_batch* batch,

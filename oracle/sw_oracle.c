@@ -394,9 +394,10 @@ int swo_choose_bruteforce(const int32_t* n_grid, int nn, const int64_t* ctx_grid
     int64_t B = dmin - now_ns;
     if (B < 0) B = 0;
     *budget_out = B;
+    /* cost(0): the decode-only iteration processes no prompt, so it is read at prefix 0 */
     int64_t t0;
     int rc = swo_cost_lookup(n_grid, nn, ctx_grid, nc, prefix_grid, np, chunk_grid, nk, cost_ns, interp,
-                             n_active, total_ctx, prefix_len, 0, &t0);
+                             n_active, total_ctx, 0, 0, &t0);
     if (rc != SWO_OK) return rc;
     if (with_margin(t0, margin_abs_ns, margin_ppm) > B) *flags_out |= SWO_F_DECODE_INFEASIBLE;
     for (int32_t c = (L / quantum) * quantum; c >= 1; c -= quantum) {

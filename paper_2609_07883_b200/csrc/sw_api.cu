@@ -68,6 +68,7 @@ struct sw_ctx {
     sw_layout layout;
     int device = 0;
     int num_sms = 0;
+    bool grid_resident = false;  // the persistent grid fits the device at once (needed by the fused append + attention launch)
     int max_chunk = 0, max_decode = 0;
     int64_t max_pages = 0;
     uint8_t* ws = nullptr;
@@ -88,6 +89,17 @@ namespace {
         cudaError_t e_ = (call);                                                                             \
         if (e_ != cudaSuccess) return sw_fail(SW_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_));  \
     } while (0)
+
+// Launching calls run on the caller's current device: a context serves the device it was created on and refuses any other
+// (its workspace, tensor maps and kernel attributes belong to that device).
+sw_status check_current_device(const sw_ctx* ctx, const char* who) {
+    int current = -1;
+    SW_CUDA(cudaGetDevice(&current));
+    if (current != ctx->device)
+        return sw_fail(SW_ERR_INVALID_ARG, "%s: the context belongs to device %d but device %d is current", who, ctx->device,
+                       current);
+    return SW_OK;
+}
 
 sw_status kv_map_for(sw_ctx* ctx, const void* pool, const sw::KvMaps** out) {
     for (auto& e : ctx->kv_maps)
@@ -202,12 +214,21 @@ sw_status sw_create(const sw_layout* layout, int device, void* workspace, size_t
     const WsLayout w = ws_layout(*layout, max_chunk, max_decode, max_pages);
     if (!workspace || workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0)
         return sw_fail(SW_ERR_WORKSPACE, "sw_create: workspace must be 256-byte aligned and hold %zu bytes", w.total);
-    SW_CUDA(cudaSetDevice(device));
     cudaDeviceProp prop;
     SW_CUDA(cudaGetDeviceProperties(&prop, device));
     if (prop.major != 10)
         return sw_fail(SW_ERR_UNSUPPORTED, "sw_create: device %d is compute capability %d.%d; this library is sm_100a only",
                        device, prop.major, prop.minor);
+    // the set-up below runs with `device` current; the caller's current device is put back before returning
+    int caller_device = device;
+    SW_CUDA(cudaGetDevice(&caller_device));
+    struct Restore {
+        int dev, want;
+        ~Restore() {
+            if (dev != want) cudaSetDevice(dev);
+        }
+    } restore{caller_device, device};
+    if (caller_device != device) SW_CUDA(cudaSetDevice(device));
     sw_ctx* ctx = new (std::nothrow) sw_ctx();
     if (!ctx) return sw_fail(SW_ERR_INVALID_ARG, "sw_create: out of host memory");
     ctx->layout = *layout;
@@ -229,6 +250,12 @@ sw_status sw_create(const sw_layout* layout, int device, void* workspace, size_t
     ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
     e = cudaMemset(ctx->ws, 0, w.pf_ml);  // control words, tickets and split-KV scratch start at zero
     if (e == cudaSuccess) e = sw::configure_kernels(layout->head_dim);
+    int per_sm = 0;
+    if (e == cudaSuccess) e = sw::mixed_attn_resident_ctas_per_sm(layout->head_dim, &per_sm);
+    // The fused launch lets CTAs wait for one another's share of the KV append, so the whole grid has to be resident.
+    // Where it would not be (fewer SMs than the properties promise cannot be seen here, but a smaller shared-memory
+    // or register budget can) sw_mixed_iteration_run issues the append as a launch of its own.
+    ctx->grid_resident = (int64_t)per_sm * prop.multiProcessorCount >= ctx->num_sms;
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         delete ctx;
@@ -252,6 +279,8 @@ sw_status sw_kv_append(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const 
     if (st != SW_OK) return st;
     if (ch.rows + batch->num_decode == 0) return SW_OK;
     if (!kv_pool || !k_new || !v_new) return sw_fail(SW_ERR_INVALID_ARG, "sw_kv_append: null tensor");
+    st = check_current_device(ctx, "sw_kv_append");
+    if (st != SW_OK) return st;
     if (((reinterpret_cast<uintptr_t>(kv_pool) | reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new)) & 15) != 0)
         return sw_fail(SW_ERR_INVALID_ARG, "sw_kv_append: tensors must be 16-byte aligned");
     sw::AppendParams p{};
@@ -287,6 +316,8 @@ sw_status run_mixed(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const voi
     if (st != SW_OK) return st;
     if (ch.rows + batch->num_decode == 0) return SW_OK;
     if (!kv_pool || !q || !out) return sw_fail(SW_ERR_INVALID_ARG, "%s: null tensor", who);
+    st = check_current_device(ctx, who);
+    if (st != SW_OK) return st;
     if (((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(k_new) |
           reinterpret_cast<uintptr_t>(v_new)) & 15) != 0)
         return sw_fail(SW_ERR_INVALID_ARG, "%s: tensors must be 16-byte aligned", who);
@@ -347,6 +378,17 @@ sw_status run_mixed(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const voi
     SW_CUDA(sw::launch_mixed_attn(l.head_dim, *kv_maps, q_map, p, ctx->num_sms, static_cast<cudaStream_t>(stream)));
     return SW_OK;
 }
+
+// Append + attention: one launch, or two where the persistent grid would not be resident at once.
+sw_status run_iteration(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const void* k_new, const void* v_new, const void* q,
+                        void* out, float* lse, void* stream, const char* who) {
+    if (ctx && !ctx->grid_resident) {
+        sw_status st = sw_kv_append(ctx, kv_pool, batch, k_new, v_new, stream);
+        if (st != SW_OK) return st;
+        return run_mixed(ctx, kv_pool, batch, nullptr, nullptr, q, out, lse, stream, who);
+    }
+    return run_mixed(ctx, kv_pool, batch, k_new, v_new, q, out, lse, stream, who);
+}
 }  // namespace
 
 sw_status sw_mixed_attn_run(sw_ctx* ctx, const void* kv_pool, const sw_batch* batch, const void* q, void* out, float* lse,
@@ -357,7 +399,7 @@ sw_status sw_mixed_attn_run(sw_ctx* ctx, const void* kv_pool, const sw_batch* ba
 sw_status sw_mixed_iteration_run(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const void* k_new, const void* v_new,
                                  const void* q, void* out, float* lse, void* stream) {
     if (!k_new || !v_new) return sw_fail(SW_ERR_INVALID_ARG, "sw_mixed_iteration_run: null tensor");
-    return run_mixed(ctx, kv_pool, batch, k_new, v_new, q, out, lse, stream, "sw_mixed_iteration_run");
+    return run_iteration(ctx, kv_pool, batch, k_new, v_new, q, out, lse, stream, "sw_mixed_iteration_run");
 }
 
 sw_status sw_mixed_iteration_host(sw_ctx* ctx, void* kv_pool, const sw_batch* hb, const void* h_q, const void* h_k_new,
@@ -431,7 +473,8 @@ sw_status probe(sw_ctx* ctx, void* const* kv_pools, int32_t layers, const sw_bat
     for (int r = -warmup; r < reps; ++r) {
         SW_CUDA(cudaEventRecord(ctx->ev0, s));
         for (int layer = 0; layer < layers; ++layer) {
-            sw_status st = run_mixed(ctx, kv_pools[layer], batch, k_new, v_new, q, out, nullptr, stream, who);
+            sw_status st = k_new ? run_iteration(ctx, kv_pools[layer], batch, k_new, v_new, q, out, nullptr, stream, who)
+                                 : run_mixed(ctx, kv_pools[layer], batch, nullptr, nullptr, q, out, nullptr, stream, who);
             if (st != SW_OK) return st;
         }
         SW_CUDA(cudaEventRecord(ctx->ev1, s));

@@ -97,6 +97,69 @@ sw_status lookup(const sw_cost_table& t, int64_t n, int64_t ctx, int64_t prefix,
     return SW_OK;
 }
 
+// Largest raw cost t whose margin still fits the budget: t + margin_abs + ceil(t * ppm / 1e6) <= B (-1 if none).
+int64_t largest_raw_cost_within(int64_t B, const sw_chooser_params& p) {
+    const __int128 room = (__int128)B - p.margin_abs_ns;
+    if (room < 0) return -1;
+    __int128 t = room * 1000000 / (1000000 + (__int128)p.margin_ppm);  // estimate; the ceiling is settled below
+    auto fits = [&](__int128 v) { return v + (v * p.margin_ppm + 999999) / 1000000 <= room; };
+    while (t >= 0 && !fits(t)) --t;
+    while (fits(t + 1)) ++t;
+    return t >= (__int128)kInf ? kInf - 1 : (int64_t)t;
+}
+
+// The search of Sec. 3.2 organised around the table instead of around the candidates.  One iteration is asked for
+// `offset` prefill tokens already (first fit; 0 for a single prefill) plus c more, c a positive multiple of q with
+// c <= K * q.  The predicted cost of offset + c tokens is constant (or, with interpolation, linear) between two
+// neighbouring points of the chunk grid, and nondecreasing from point to point.  So: (1) bisect over the grid POINTS
+// that the candidates can round up to for the last one whose cost plus margin meets the budget B; (2) every candidate up
+// to that point is feasible; with interpolation the stretch towards the next point may hold more, and the last
+// feasible token count there follows from one division; (3) the answer is the largest candidate not beyond that.
+// Returns c (0 when no candidate is feasible); *predicted is set to the cost plus margin at the answer when c > 0.
+// By Proposition 1 this is the maximiser of Eq. (1); the parity tests compare it with the exhaustive scan.
+sw_status largest_feasible(const sw_cost_table& t, const sw_chooser_params& params, int64_t n, int64_t ctx, int64_t prefix,
+                           int64_t offset, int32_t K, int32_t q, int64_t B, int32_t* c_out, int64_t* predicted,
+                           int32_t* queries) {
+    *c_out = 0;
+    if (K <= 0) return SW_OK;
+    const size_t a = round_up_index(t.n_grid, n);
+    const size_t b = round_up_index(t.ctx_grid, ctx);
+    const size_t p = round_up_index(t.prefix_grid, prefix);
+    if (a == t.n_grid.size() || b == t.ctx_grid.size() || p == t.prefix_grid.size())
+        return sw_fail(SW_ERR_OUT_OF_RANGE, "cost lookup: n=%lld ctx=%lld prefix=%lld beyond the table grid", (long long)n,
+                       (long long)ctx, (long long)prefix);
+    const int64_t* row = &t.cost[t.at(a, b, p, 0)];
+    const std::vector<int32_t>& grid = t.chunk_grid;
+    const int64_t nk = (int64_t)grid.size();
+    const int64_t x_first = offset + q, x_last = offset + (int64_t)K * q;   // smallest and largest candidate total
+    const int64_t raw_max = largest_raw_cost_within(B, params);            // a raw cost fits iff it is <= raw_max
+    // grid points the candidates round up to: [ea, eb]; index nk stands for "beyond the grid" (infinite cost)
+    const int64_t ea = (int64_t)round_up_index(grid, x_first), eb = (int64_t)round_up_index(grid, x_last);
+    int64_t lo = ea - 1, hi = eb;  // invariant: points <= lo fit (or lo == ea - 1), points > hi do not
+    while (lo < hi) {
+        const int64_t mid = lo + (hi - lo + 1) / 2;
+        *queries += 1;
+        if (mid < nk && row[mid] <= raw_max) lo = mid; else hi = mid - 1;
+    }
+    int64_t x_best = lo >= ea ? (lo == nk ? x_last : std::min<int64_t>(grid[(size_t)lo], x_last)) : 0;  // 0: none so far
+    if (lo == eb && lo < nk) x_best = x_last;  // the last candidate itself rounds up to a point that fits
+    if (t.interp && x_best < x_last && lo >= 0 && lo + 1 < nk && row[lo] <= raw_max) {
+        // between grid[lo] and grid[lo + 1]: cost = row[lo] + ceil((row[lo+1] - row[lo]) * dx / span) <= raw_max
+        const int64_t rise = row[lo + 1] - row[lo], span = (int64_t)grid[(size_t)lo + 1] - grid[(size_t)lo];
+        const __int128 room = (__int128)raw_max - row[lo];
+        const int64_t dx = rise <= 0 ? span : (int64_t)std::min<__int128>(span, room * span / rise);
+        x_best = std::max(x_best, std::min<int64_t>(grid[(size_t)lo] + dx, x_last));
+    }
+    if (x_best < x_first) return SW_OK;
+    const int32_t c = (int32_t)((x_best - offset) / q) * q;
+    int64_t raw = 0;
+    sw_status st = lookup(t, n, ctx, prefix, offset + c, &raw);
+    if (st != SW_OK) return st;
+    *c_out = c;
+    *predicted = add_margin(raw, params);
+    return SW_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -159,59 +222,17 @@ sw_status sw_choose_chunk(const sw_cost_table* table, const sw_chooser_params* p
     if (n_active < 0 || remaining_prefill < 0 || prefix_len < 0 || total_ctx < 0 || params->c_max < 0 ||
         params->margin_ppm < 0 || params->margin_abs_ns < 0 || (n_active > 0 && !deadlines_ns))
         return sw_fail(SW_ERR_INVALID_ARG, "sw_choose_chunk: negative size or missing deadlines");
-    const int32_t q = params->chunk_quantum > 1 ? params->chunk_quantum : 1;
-    *out = sw_choice{0, 0, 0, 0, 0};
-    // P empty -> 0
-    if (remaining_prefill == 0) {
-        out->flags = SW_F_NO_PREFILL;
-        return SW_OK;
-    }
-    // L = min(C_max, remaining(r))
-    const int32_t L = std::min(params->c_max, remaining_prefill);
-    if (params->c_max < remaining_prefill) out->flags |= SW_F_CAPPED;
-    // A empty -> L
-    if (n_active == 0) {
-        out->chunk = L - L % q;
-        out->flags |= SW_F_NO_DECODE;
-        return SW_OK;
-    }
-    if (!table) return sw_fail(SW_ERR_INVALID_ARG, "sw_choose_chunk: a cost table is required when decodes are active");
-    // B = min_i (l_i + D - s), clamped at zero (Sec. 3.1)
-    const int64_t earliest = *std::min_element(deadlines_ns, deadlines_ns + n_active);
-    const int64_t B = earliest > now_ns ? earliest - now_ns : 0;
-    out->budget_ns = B;
-
-    int64_t t_raw = 0;
-    sw_status st = lookup(*table, n_active, total_ctx, prefix_len, 0, &t_raw);
-    if (st != SW_OK) return st;
-    const int64_t decode_only = add_margin(t_raw, *params);
-    if (decode_only > B) out->flags |= SW_F_DECODE_INFEASIBLE;
-    out->predicted_ns = decode_only;
-
-    // upper-mid bisection over k in [0, L/q], candidate chunk c = k*q
-    int32_t lo = 0, hi = L / q;
-    int64_t predicted_at_lo = decode_only;
-    while (lo < hi) {
-        const int32_t mid = lo + (hi - lo + 1) / 2;
-        st = lookup(*table, n_active, total_ctx, prefix_len, (int64_t)mid * q, &t_raw);
-        if (st != SW_OK) return st;
-        out->queries += 1;
-        const int64_t t = add_margin(t_raw, *params);
-        if (t <= B) {
-            lo = mid;
-            predicted_at_lo = t;
-        } else {
-            hi = mid - 1;
-        }
-    }
-    out->chunk = lo * q;
-    out->predicted_ns = predicted_at_lo;
-    return SW_OK;
+    // Sec. 3.2 / Algorithm 1 as one call of the first-fit routine with a single pending request: nothing pending gives
+    // 0, no active decode gives the capped remainder, otherwise the largest chunk whose predicted cost meets the budget.
+    int32_t chunk = 0, count = 0;
+    return sw_choose_chunks(table, params, now_ns, deadlines_ns, n_active, total_ctx, &prefix_len, &remaining_prefill, 1, &chunk,
+                            &count, out);
 }
 
-// Several prefills per iteration by first fit: requests oldest first, each admitted whole while the prediction for the
-// total still meets the budget; the first one that does not fit whole is cut by the bisection of Algorithm 1 and ends
-// the list.
+// Several prefills per iteration by first fit (Sec. 3.3): requests oldest first, each admitted whole while the
+// prediction for the total still meets the budget; the first one that does not fit whole gets the largest feasible part
+// and ends the list.  A decode-only iteration processes no prompt, so its cost (the c = 0 column, which decides
+// SW_F_DECODE_INFEASIBLE) is read at prefix 0 whatever the pending requests' prefixes are.
 sw_status sw_choose_chunks(const sw_cost_table* table, const sw_chooser_params* params, int64_t now_ns,
                            const int64_t* deadlines_ns, int32_t n_active, int64_t total_ctx, const int32_t* prefix_lens,
                            const int32_t* remaining_prefill, int32_t num_pending, int32_t* chunks, int32_t* num_chunks,
@@ -231,11 +252,12 @@ sw_status sw_choose_chunks(const sw_cost_table* table, const sw_chooser_params* 
         out->flags = SW_F_NO_PREFILL;
         return SW_OK;
     }
+    if (params->c_max < remaining_prefill[0]) out->flags |= SW_F_CAPPED;
     int64_t B = 0;
     if (n_active > 0) {
         if (!table) return sw_fail(SW_ERR_INVALID_ARG, "sw_choose_chunks: a cost table is required when decodes are active");
         const int64_t earliest = *std::min_element(deadlines_ns, deadlines_ns + n_active);
-        B = earliest > now_ns ? earliest - now_ns : 0;
+        B = earliest > now_ns ? earliest - now_ns : 0;   // the clamp of Sec. 3.1
         out->budget_ns = B;
         int64_t t_raw = 0;
         sw_status st = lookup(*table, n_active, total_ctx, 0, 0, &t_raw);
@@ -252,31 +274,16 @@ sw_status sw_choose_chunks(const sw_cost_table* table, const sw_chooser_params* 
         const int64_t room = (int64_t)params->c_max - tokens;
         const int32_t L = (int32_t)std::min<int64_t>(room, remaining_prefill[j]);
         if (L <= 0) break;
-        if ((int64_t)params->c_max - tokens < remaining_prefill[j]) out->flags |= SW_F_CAPPED;
+        if (room < remaining_prefill[j]) out->flags |= SW_F_CAPPED;
         int32_t c = 0;
         if (n_active == 0) {
-            c = L - L % q;
+            c = L - L % q;   // no deadline to meet: the table is not consulted
         } else {
-            const int64_t prefix = prefix_sum + prefix_lens[j];
-            // upper-mid bisection over k in [0, L/q], c = k*q (Algorithm 1 with the tokens admitted so far as offset)
-            int32_t lo = 0, hi = L / q;
-            int64_t predicted_at_lo = out->predicted_ns;
-            while (lo < hi) {
-                const int32_t mid = lo + (hi - lo + 1) / 2;
-                int64_t t_raw = 0;
-                sw_status st = lookup(*table, n_active, total_ctx, prefix, tokens + (int64_t)mid * q, &t_raw);
-                if (st != SW_OK) return st;
-                out->queries += 1;
-                const int64_t t = add_margin(t_raw, *params);
-                if (t <= B) {
-                    lo = mid;
-                    predicted_at_lo = t;
-                } else {
-                    hi = mid - 1;
-                }
-            }
-            c = lo * q;
-            if (c > 0) out->predicted_ns = predicted_at_lo;
+            int64_t predicted = 0;
+            sw_status st = largest_feasible(*table, *params, n_active, total_ctx, prefix_sum + prefix_lens[j], tokens, L / q, q, B,
+                                            &c, &predicted, &out->queries);
+            if (st != SW_OK) return st;
+            if (c > 0) out->predicted_ns = predicted;
         }
         if (c == 0) break;
         chunks[*num_chunks] = c;

@@ -125,6 +125,7 @@ cudaError_t launch_kv_append(const AppendParams& p, cudaStream_t stream);
 cudaError_t launch_mixed_attn(int head_dim, const KvMaps& kv_maps, const CUtensorMap& q_map, const MixedParams& p,
                               int num_sms, cudaStream_t stream);
 cudaError_t configure_kernels(int head_dim);
+cudaError_t mixed_attn_resident_ctas_per_sm(int head_dim, int* out);
 cudaError_t launch_selftest_wait(int32_t* ctrl, long long budget_cycles, cudaStream_t stream);
 size_t mixed_attn_smem_bytes(int head_dim);
 

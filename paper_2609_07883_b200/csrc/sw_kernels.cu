@@ -563,9 +563,12 @@ __device__ bool run_unit(const CUtensorMap* kvp_map, const MixedParams& p, const
             const int pi = pg0 + issued + lane;
             ids = pi < pg1 ? u.pages[pi] : 0;
         }
-        const int page = __shfl_sync(0xffffffffu, ids, issued & 31);
+        int page = __shfl_sync(0xffffffffu, ids, issued & 31);
         if (page < 0 || (int64_t)page >= p.num_pages) {
+            // a bad id never reaches the copy engine: the problem is reported and page 0 is fetched in its place, so
+            // the barrier still receives the bytes it expects
             if (lane == 0) report(p.ctrl, SW_ERR_OUT_OF_RANGE, kSiteAttnPage, u.q_row);
+            page = 0;
         }
         // the request's last page holds the row this iteration appends
         if (p.pool != nullptr && (pg0 + issued + 1) * kPageSize >= u.len && !wait_append(p)) {
@@ -1000,6 +1003,25 @@ cudaError_t configure_kernels(int head_dim) {
     e = cudaFuncSetAttribute(sw_mixed_attn_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(sw_mixed_attn_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+
+// CTAs of the persistent kernel that one SM can hold at a time (the smaller figure of the two forms).  The fused launch
+// makes CTAs wait for one another's share of the KV append, which is only safe when the whole grid is resident.
+cudaError_t mixed_attn_resident_ctas_per_sm(int head_dim, int* out) {
+    const size_t bytes = mixed_attn_smem_bytes(head_dim);
+    int a = 0, b = 0;
+    cudaError_t e;
+    if (head_dim == 64) {
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, sw_mixed_attn_kernel<64, false>, kThreads, bytes);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, sw_mixed_attn_kernel<64, true>, kThreads, bytes);
+    } else {
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, sw_mixed_attn_kernel<128, false>, kThreads, bytes);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, sw_mixed_attn_kernel<128, true>, kThreads, bytes);
+    }
+    *out = a < b ? a : b;
+    return e;
 }
 
 cudaError_t launch_mixed_attn(int head_dim, const KvMaps& kv_maps, const CUtensorMap& q_map, const MixedParams& p,

@@ -351,7 +351,13 @@ __device__ __forceinline__ bool pf_produce(const CUtensorMap* kv_map, const CUte
     }
     const int npages = (pf_chunk<D, kMulti>(p, sh, 0, it.chunk) + pf_chunk<D, kMulti>(p, sh, 1, it.chunk) + kPageSize - 1) / kPageSize;
     auto page_of = [&](int j) {
-        return (lane < 8 && j * 8 + lane < npages) ? p.prefill_pages[pf_chunk<D, kMulti>(p, sh, 3, it.chunk) + j * 8 + lane] : 0;
+        int id = (lane < 8 && j * 8 + lane < npages) ? p.prefill_pages[pf_chunk<D, kMulti>(p, sh, 3, it.chunk) + j * 8 + lane] : 0;
+        if (id < 0 || (int64_t)id >= p.num_pages) {
+            // reported, and page 0 fetched in its place: a bad id never reaches the copy engine
+            report(p.ctrl, SW_ERR_OUT_OF_RANGE, kSiteAttnPage, it.item);
+            id = 0;
+        }
+        return id;
     };
     int id_next = page_of(it.j0);
     for (int j = it.j0; j < it.j1; ++j, ++kv_it) {

@@ -51,12 +51,17 @@ DeviceState g_devices[kMaxDevices];
         if (e_ != cudaSuccess) return sw_fail(SW_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_));  \
     } while (0)
 
-// Once per device, with that device current.
+// Every call: `device` must be the caller's current device (the launch, the clearing of the scratch and the address of
+// the scratch all belong to the current device; nothing here changes it).  Once per device: the set-up below.
 sw_status setup_device(int device, DeviceState** out) {
     if (device < 0 || device >= kMaxDevices) return sw_fail(SW_ERR_INVALID_ARG, "device index %d out of range", device);
+    int current = -1;
+    SW_CUDA(cudaGetDevice(&current));
+    if (current != device)
+        return sw_fail(SW_ERR_INVALID_ARG, "sw_decode_attn_static: device %d was named but device %d is current", device,
+                       current);
     DeviceState& st = g_devices[device];
     if (!st.ready) {
-        SW_CUDA(cudaSetDevice(device));
         cudaDeviceProp prop;
         SW_CUDA(cudaGetDeviceProperties(&prop, device));
         if (prop.major != 10)

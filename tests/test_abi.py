@@ -58,3 +58,24 @@ def test_host_side_argument_errors_without_a_gpu(lib_path):
     with pytest.raises(B.SwError) as e:
         B.CostTable([2, 1], [10], [0], [0, 16], [1, 2, 3, 4])
     assert e.value.status == B.SW_ERR_INVALID_ARG
+
+
+def test_static_entry_point_refuses_bad_arguments_before_any_cuda_call(lib_path):
+    """Host-side refusals of sw_decode_attn_static: they come before the first CUDA call, so they can be checked here."""
+    import ctypes as C
+
+    from paper_2609_07883_b200 import binding as B
+    from paper_2609_07883_b200 import workloads as W
+
+    fake = 0x1000  # aligned, never dereferenced: every call below is refused on its arguments
+    lay = B.make_layout(W.AttnShape(8, 2, 128), 64)
+    one = B.sw_batch(0, 0, None, 0, 1, fake, fake, fake, 0, None, None, None)
+    call = lambda layout, device, batch: B._lib.sw_decode_attn_static(C.byref(layout), device, fake, C.byref(batch), fake,
+                                                                      fake, None, None)
+    assert call(lay, -1, one) == B.SW_ERR_INVALID_ARG and "out of range" in B.sw_last_error()
+    assert call(lay, 64, one) == B.SW_ERR_INVALID_ARG
+    too_many = B.sw_batch(0, 0, None, 0, B.SW_STATIC_MAX_DECODE + 1, fake, fake, fake, 0, None, None, None)
+    assert call(lay, 0, too_many) == B.SW_ERR_WORKSPACE and "static limit" in B.sw_last_error()
+    chunked = B.sw_batch(0, 16, fake, 1, 1, fake, fake, fake, 0, None, None, None)
+    assert call(lay, 0, chunked) == B.SW_ERR_UNSUPPORTED
+    assert call(B.make_layout(W.AttnShape(32, 16, 128), 64), 0, one) == B.SW_ERR_WORKSPACE   # more than 8 KV heads

@@ -224,8 +224,48 @@ def test_bad_page_ids_are_reported_not_faulted(gpu, oracle):
     r2 = gpu.Runner(bad2, t)
     r2.append()
     assert r2.status()[0] == r2.B.SW_ERR_OUT_OF_RANGE
+    # the same bad prompt page id in the attention call: the chunk-prefill producer reports it and reads page 0 in its
+    # place (no out-of-range coordinate reaches the copy engine); likewise for ids whose doubled value would wrap
+    for bad_id in (-3, batch.num_pages, (1 << 30) + 1, -(1 << 30) - 7):
+        bad3 = W.MixedBatch(**{**batch.__dict__})
+        bad3.prefill_pages = batch.prefill_pages.copy()
+        bad3.prefill_pages[0] = bad_id
+        r3 = gpu.Runner(bad3, t)
+        r3.attend()
+        assert r3.status()[0] == r3.B.SW_ERR_OUT_OF_RANGE, bad_id
+        assert r3.status() == (0, 0)
+        bad4 = W.MixedBatch(**{**batch.__dict__})
+        bad4.decode_pages = batch.decode_pages.copy()
+        bad4.decode_pages[0] = bad_id
+        r4 = gpu.Runner(bad4, t)
+        r4.attend()
+        assert r4.status()[0] == r4.B.SW_ERR_OUT_OF_RANGE, bad_id
     # a good iteration on the same context still works afterwards
     run_and_compare(gpu, oracle, batch, t, what="after bad ids")
+
+
+def test_calls_refuse_a_context_of_another_device(gpu):
+    """A context serves the device it was created on: with another device named or current the launching calls return
+    SW_ERR_INVALID_ARG and launch nothing.  (One GPU is enough: the static entry point is told a device that is not
+    the current one.)"""
+    import torch
+
+    from paper_2609_07883_b200 import binding as B
+
+    rng = np.random.default_rng(41)
+    batch = W.make_batch(W.TINY, 64, [40], 0, 0, rng)
+    t = W.host_tensors(batch, rng)
+    r = gpu.Runner(batch, t)
+    with pytest.raises(B.SwError) as e:
+        B.sw_decode_attn_static(B.make_layout(W.TINY, 64), 1, r.pool, r.dbatch, r.q, r.out)
+    assert e.value.status == B.SW_ERR_INVALID_ARG and "is current" in str(e.value)
+    if torch.cuda.device_count() > 1:
+        with torch.cuda.device(1):
+            with pytest.raises(B.SwError) as e:
+                B.sw_mixed_attn_run(r.ctx, r.pool, r.dbatch, r.q, r.out)
+            assert e.value.status == B.SW_ERR_INVALID_ARG and "is current" in str(e.value)
+    # creating a context leaves the caller's current device as it was
+    assert torch.cuda.current_device() == 0
 
 
 def test_host_argument_errors(gpu):

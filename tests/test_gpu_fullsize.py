@@ -22,38 +22,8 @@ def gpu():
     return gpu_util
 
 
-def run_case(gpu, oracle, batch, pairs, seed, what):
-    import torch
-
-    from paper_2609_07883_b200 import binding as B
-
-    dev = torch.device("cuda", 0)
-    sh = batch.shape
-    total_pages = int(batch.prefill_pages.shape[0] + batch.decode_pages.shape[0])
-    ctx = B.Context(sh, batch.num_pages, max(batch.chunk_len, 1), max(batch.num_decode, 1), total_pages + 16)
-    db = B.DeviceBatch(batch, dev)
-    pool = torch.empty(batch.num_pages * sh.page_elems, dtype=torch.bfloat16, device=dev)
-    W.fill_normal_bf16_(pool, seed)
-    gen = torch.Generator(device=dev)
-    gen.manual_seed(seed + 1)
-    R = batch.num_rows
-    q = torch.randn(R, sh.num_q_heads, sh.head_dim, device=dev, generator=gen).to(torch.bfloat16)
-    k_new = torch.randn(R, sh.num_kv_heads, sh.head_dim, device=dev, generator=gen).to(torch.bfloat16)
-    v_new = torch.randn(R, sh.num_kv_heads, sh.head_dim, device=dev, generator=gen).to(torch.bfloat16)
-    out = torch.zeros_like(q)
-    lse = torch.zeros(R, sh.num_q_heads, dtype=torch.float32, device=dev)
-    host_pool = gpu.torch_to_bits(pool)          # the inputs, before the append
-    B.sw_kv_append(ctx, pool, db, k_new, v_new)
-    B.sw_mixed_attn_run(ctx, pool, db, q, out, lse)
-    torch.cuda.synchronize()
-    assert B.sw_check_status(ctx, raise_on_error=False) == (0, 0)
-    assert oracle.kv_append(host_pool, batch, gpu.torch_to_bits(k_new), gpu.torch_to_bits(v_new)) == 0
-    assert np.array_equal(gpu.torch_to_bits(pool), host_pool), f"{what}: pool differs after append"
-    pairs = np.asarray(pairs, dtype=np.int32)
-    ref, ref_lse, _ = oracle.mixed_attention(host_pool, batch, gpu.torch_to_bits(q), pairs=pairs)
-    got = W.bf16_bits_to_f64(gpu.torch_to_bits(out))[pairs[:, 0], pairs[:, 1]]
-    got_lse = lse.cpu().numpy().astype(np.float64)[pairs[:, 0], pairs[:, 1]]
-    return gpu.compare(got, got_lse, ref, ref_lse, what)
+def run_case(gpu, oracle, batch, pairs, seed, what, **kw):
+    return gpu.run_device_case(oracle, batch, pairs, seed, what, **kw)
 
 
 def sample_pairs(batch, rng, chunk_rows, n_decode_extra):
@@ -85,6 +55,38 @@ def test_long_context_workload(gpu, oracle):
     batch = W.long_batch(1024, 98304, n=16, rng=rng)
     pairs = sample_pairs(batch, np.random.default_rng(3), [0, 1, 63, 64, 512, 1023], 6)
     run_case(gpu, oracle, batch, pairs, 103, "long n=16 C=1024 P=98304")
+
+
+def edge_pairs(gpu, batch, rng, n_decode_extra):
+    """(row, head) sample of a large case: the chunk rows next to every tile, KV-tile and (sampled) page edge, the
+    shortest and the longest decode and a few more, one random query head each."""
+    return sample_pairs(batch, rng, gpu.boundary_rows(batch.chunk_len, batch.shape.group), n_decode_extra)
+
+
+@pytest.mark.parametrize("C", [2048, 4096])
+def test_prefill_only_large_chunk_at_prefix_zero(gpu, oracle, C):
+    """The chunk sizes the tensor-core target is stated on, at prefix 0: 256 / 512 work items of 1 to 32 KV tiles, pulled
+    longest first from the counter over several waves."""
+    batch = W.make_batch(W.LLAMA, C // 16 + 64, [], 0, C, np.random.default_rng(40 + C))
+    run_case(gpu, oracle, batch, edge_pairs(gpu, batch, np.random.default_rng(5), 0), 140 + C, f"prefill-only C={C} P=0")
+
+
+def test_mixed_workload_large_chunk_fused(gpu, oracle):
+    """C=4096 at prefix 28672 beside the 128 log-normal decodes, append and attention in one launch."""
+    batch = W.mixed_batch(4096, 28672, n=128, rng=W.rng_for(2))
+    run_case(gpu, oracle, batch, edge_pairs(gpu, batch, np.random.default_rng(6), 16), 104,
+             "mixed n=128 C=4096 P=28672 (fused)", fused=True)
+
+
+def test_long_context_workload_large_chunks(gpu, oracle):
+    """C=8192 and C=4096 at prefix 98304 beside the 16 decodes of 32k-131k tokens (the largest single-GPU configuration,
+    and the one bench.py times by default): 1024 / 512 work items of about 800 KV tiles each."""
+    import dataclasses
+
+    big = W.long_batch(8192, 98304, n=16, rng=W.rng_for(3))
+    run_case(gpu, oracle, big, edge_pairs(gpu, big, np.random.default_rng(7), 4), 105, "long n=16 C=8192 P=98304", fused=True)
+    half = dataclasses.replace(big, chunk_len=4096)
+    run_case(gpu, oracle, half, edge_pairs(gpu, half, np.random.default_rng(8), 4), 106, "long n=16 C=4096 P=98304")
 
 
 def test_page_ids_above_two_to_the_twenty(gpu, oracle):

@@ -94,7 +94,7 @@ def test_mixed_iteration_with_long_prefix_and_decodes(gpu, oracle):
     full_compare(gpu, oracle, batch, W.host_tensors(batch, rng), "mixed long prefix")
 
 
-def test_dominant_key_and_constant_v_closed_forms(gpu, oracle):
+def test_constant_v_and_causal_closed_forms(gpu, oracle):
     import torch
 
     rng = np.random.default_rng(79)
