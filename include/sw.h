@@ -225,7 +225,7 @@ typedef struct {
     int32_t flags;        /* SW_F_* */
     int64_t budget_ns;    /* B = max(0, min_i d_i - now) */
     int64_t predicted_ns; /* T^ + delta at the chosen chunk (INT64_MAX never; 0 when no table query was made) */
-    int32_t queries;      /* cost-model queries made by the bisection */
+    int32_t queries;      /* table reads made by the bisection */
 } sw_choice;
 
 /* Several prefills in one iteration by first fit (Sec. 3.3, "Prefill batching").  The pending requests are given
@@ -279,9 +279,15 @@ sw_status sw_telemetry_exceeds(const sw_telemetry* t, int32_t n, int32_t c, int3
 sw_status sw_telemetry_reset(sw_telemetry* t);
 sw_status sw_telemetry_get_totals(const sw_telemetry* t, sw_telemetry_totals* out);
 
-/* Algorithm 1: P empty -> 0; L = min(C_max, remaining); A empty -> L; B = min_i(d_i) - now; upper-mid
- * bisection over [0, L] on T^ + delta <= B.  deadlines_ns are absolute next-token deadlines d_i = l_i + D_i
- * (HOST array, n_active entries).  remaining_prefill = 0 means no pending prefill. */
+/* The chunk decision of one iteration (Sec. 3.1-3.2, Eq. (1), Algorithm 1): the largest chunk c <= min(C_max,
+ * remaining_prefill) whose predicted cost T^(n_active, total_ctx, prefix_len, c) + delta still ends before the
+ * earliest of the active decodes' next-token deadlines.  deadlines_ns are absolute deadlines d_i = l_i + D_i (HOST
+ * array, n_active entries), so the budget is B = max(0, min_i d_i - now_ns).  Nothing pending (remaining_prefill == 0)
+ * gives 0; no active decode gives the capped remainder without a table.  The cost is nondecreasing in c, so the
+ * answer is found by bisection (Proposition 1); this implementation bisects over the points of the table's chunk
+ * grid and closes the last stretch in closed form, which needs at most ceil(log2(candidates + 1)) table reads.
+ * The decode-only cost (c = 0), which decides SW_F_DECODE_INFEASIBLE, is read at prefix 0: an iteration without
+ * prefill tokens processes no prompt. */
 sw_status sw_choose_chunk(const sw_cost_table* table, const sw_chooser_params* params, int64_t now_ns,
                           const int64_t* deadlines_ns, int32_t n_active, int64_t total_ctx, int32_t prefix_len,
                           int32_t remaining_prefill, sw_choice* out);

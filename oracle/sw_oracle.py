@@ -22,19 +22,27 @@ F_NO_PREFILL, F_NO_DECODE, F_DECODE_INFEASIBLE, F_CAPPED = 1, 2, 4, 8
 INF = (1 << 63) - 1
 
 
-def build(force: bool = False) -> Path:
-    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
-        tmp = _LIB.with_suffix(f".{os.getpid()}.tmp")
-        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fopenmp", "-shared", "-fPIC", "-o", str(tmp),
-                               str(_SRC), "-lm"])
-        os.replace(tmp, _LIB)
-    return _LIB
+# SW_ORACLE_SANITIZE=1 builds and loads the same source instrumented with -fsanitize=address,undefined (the sanitizer
+# run of the CPU tests; the process must have been started with the sanitizer runtimes preloaded).
+_SANITIZE = os.environ.get("SW_ORACLE_SANITIZE", "") not in ("", "0")
+_LIB_ASAN = _HERE / "libsw_oracle_asan.so"
+
+
+def build(force: bool = False, sanitize: bool = False) -> Path:
+    target = _LIB_ASAN if sanitize else _LIB
+    flags = (["-O1", "-g", "-fsanitize=address,undefined", "-fno-sanitize-recover=undefined", "-fno-omit-frame-pointer"]
+             if sanitize else ["-O2"])
+    if force or not target.exists() or target.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = target.with_suffix(f".{os.getpid()}.tmp")
+        subprocess.check_call(["gcc"] + flags + ["-std=c11", "-fopenmp", "-shared", "-fPIC", "-o", str(tmp), str(_SRC), "-lm"])
+        os.replace(tmp, target)
+    return target
 
 
 def lib():
     global _lib
     if _lib is None:
-        _lib = C.CDLL(str(build()))
+        _lib = C.CDLL(str(build(sanitize=_SANITIZE)))
         _lib.swo_pool_index.restype = C.c_int64
         _lib.swo_pool_index.argtypes = [C.c_int64] + [C.c_int] * 7
         _lib.swo_analytic_cost_ns.restype = C.c_int64

@@ -13,7 +13,8 @@ import numpy as np
 
 import os
 
-# SLOWEAVE_LIB overrides the library file (used to compare differently tuned builds of the same sources)
+# SLOWEAVE_LIB names another build of the same library to load instead of the default file: the sanitizer run of the
+# CPU tests loads ``libsloweave_asan.so`` (``build.build_sanitized()``) this way.
 _LIB_PATH = Path(os.environ.get("SLOWEAVE_LIB") or Path(__file__).resolve().parent / "libsloweave.so")
 if not _LIB_PATH.exists():
     raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2609_07883_b200.build` "

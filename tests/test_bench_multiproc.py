@@ -53,12 +53,12 @@ def test_single_process_is_the_identity():
 
 def test_reference_arm_prints_only_on_rank_zero():
     env = dict(os.environ, RANK="1", LOCAL_RANK="1", WORLD_SIZE="2")
-    r = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "0"],
-                       env=env, capture_output=True, text=True, timeout=120)
+    r = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--impl", "reference", "--workload", "chat", "--steps", "1",
+                        "--warmup", "0"], env=env, capture_output=True, text=True, timeout=120)
     assert r.returncode == 0 and r.stdout.strip() == ""
     env0 = dict(os.environ, RANK="0", LOCAL_RANK="0", WORLD_SIZE="2")
-    r0 = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "0",
-                         "--ref-budget-keys", "200000"], env=env0, capture_output=True, text=True, timeout=300)
+    r0 = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--impl", "reference", "--workload", "chat", "--steps", "1",
+                         "--warmup", "0", "--ref-seconds", "0.05"], env=env0, capture_output=True, text=True, timeout=300)
     line = json.loads(r0.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["unit"] == "us" and line["higher_is_better"] is False
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0

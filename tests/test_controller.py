@@ -169,3 +169,22 @@ def test_first_fit_over_several_pending_requests_matches_the_oracle(B, oracle):
                 one = B.sw_choose_chunk(lt, now, dl, ctx, prefixes[0], remaining[0], c_max=c_max, chunk_quantum=quantum,
                                         margin_abs_ns=mabs, margin_ppm=mppm)
                 assert ([one.chunk] if one.chunk else []) == got and one.predicted_ns == ch.predicted_ns
+
+
+def test_decode_only_cost_is_read_at_prefix_zero(B, oracle):
+    """A table whose c = 0 column differs between prefix points: an iteration without prefill tokens processes no prompt,
+    so both entry points (and the exhaustive scan) judge SW_F_DECODE_INFEASIBLE by the cost at prefix 0, and agree."""
+    grids = ([4], [1000], [0, 100], [0, 16], np.array([10, 20, 50, 60], dtype=np.int64))
+    lt, ot = both_tables(B, oracle, *grids)
+    one = B.sw_choose_chunk(lt, 0, [30] * 4, 1000, 100, 64)
+    many, ch = B.sw_choose_chunks(lt, 0, [30] * 4, 1000, [100], [64])
+    want = ot.choose(0, [30] * 4, 1000, 100, 64)
+    assert want == (0, 0, 30)
+    assert (one.chunk, one.flags, one.budget_ns, one.predicted_ns) == (0, 0, 30, 10)
+    assert many == [] and (ch.chunk, ch.flags, ch.budget_ns, ch.predicted_ns) == (0, 0, 30, 10)
+    # at prefix 0 the 16-token chunk costs 20 and fits; at prefix 100 it costs 60 and does not
+    assert B.sw_choose_chunk(lt, 0, [30] * 4, 1000, 0, 64).chunk == 16
+    # below the decode-only cost the flag is raised, by all three
+    assert B.sw_choose_chunk(lt, 0, [9] * 4, 1000, 100, 64).flags == B.SW_F_DECODE_INFEASIBLE
+    assert B.sw_choose_chunks(lt, 0, [9] * 4, 1000, [100], [64])[1].flags == B.SW_F_DECODE_INFEASIBLE
+    assert ot.choose(0, [9] * 4, 1000, 100, 64) == (0, B.SW_F_DECODE_INFEASIBLE, 9)
