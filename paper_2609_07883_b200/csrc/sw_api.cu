@@ -34,6 +34,7 @@ bool layout_supported(const sw_layout& l) {
     const int g = l.num_q_heads / l.num_kv_heads;
     if (!(g == 1 || g == 2 || g == 4 || g == 8)) return false;
     if (l.num_pages > (int64_t)1 << 30) return false;
+    if (2 * l.num_pages * l.num_kv_heads >= (int64_t)1 << 31) return false;  // (page, K|V, head) blocks are int32 coordinates
     return true;
 }
 
@@ -364,7 +365,7 @@ sw_status run_mixed(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const voi
     p.pf_tickets = reinterpret_cast<int32_t*>(ctx->ws + ctx->w.pf_tickets);
     // q as [row][head][element] restricted to the chunk rows: one box = 128 tile rows (token-major, the g heads of a
     // KV head minor) x 64 elements; rows past the chunk read as zero
-    CUtensorMap q_map = kv_maps->tile;
+    CUtensorMap q_map = kv_maps->half;
     if (p.C > 0) {
         const cuuint64_t dims[3] = {(cuuint64_t)l.head_dim, (cuuint64_t)l.num_q_heads, (cuuint64_t)p.C};
         const cuuint64_t strides[2] = {(cuuint64_t)l.head_dim * 2, (cuuint64_t)l.num_q_heads * l.head_dim * 2};

@@ -84,13 +84,15 @@ struct AppendParams {
     int32_t* ctrl;
 };
 
-// Tensor maps of one KV pool [page][K|V][kv head][slot][element].
-//   tile: 4-D {element, slot, K|V x kv head, page}, box = [16 slots][64 elements], one 128-byte-swizzled block; the
-//         chunk-prefill producer lays such blocks out as 128-key MMA operand tiles.
-//   page: 5-D {element % 64, slot, element / 64, 2 * page + K|V, kv head}, box = all of one head's K and V in a page
-//         (2 x head_dim/64 blocks of the same swizzled form, K blocks first): a decode unit fetches a page with one copy.
+// Tensor maps of one KV pool [page][K|V][kv head][slot][element].  A (page, K|V, kv head) block of 16 slots x head_dim
+// elements reads as head_dim/64 x 2 swizzle atoms of [8 slots][64 elements] (1 KB each in shared memory).
+//   half: 5-D {element % 64, slot % 8, element / 64, slot / 8, block} with block = (2 * page + K|V) * Hkv + kv head; box = one
+//         block, landing as [slot group][64-element block][8][128 B]: the chunk-prefill producer fetches the eight pages
+//         of a 128-key operand tile with eight such copies (one per page, K and V separately).
+//   page: 5-D {element % 64, slot, element / 64, 2 * page + K|V, kv head}; box = all of one head's K and V in a page, as
+//         2 x head_dim/64 blocks of [16][128 B], K blocks first: a decode unit fetches a page with one copy.
 struct KvMaps {
-    CUtensorMap tile;
+    CUtensorMap half;
     CUtensorMap page;
 };
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -102,11 +104,10 @@ inline CUresult encode_kv_maps(EncodeTiledFn encode, const sw_layout& l, const v
     const cuuint64_t side = (cuuint64_t)l.num_kv_heads * head;         // all K (or all V) of a page
     const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
     {
-        const cuuint64_t dims[4] = {(cuuint64_t)l.head_dim, (cuuint64_t)kPageSize, (cuuint64_t)2 * l.num_kv_heads,
-                                    (cuuint64_t)l.num_pages};
-        const cuuint64_t strides[3] = {row, head, 2 * side};
-        const cuuint32_t box[4] = {64, (cuuint32_t)kPageSize, 1, 1};
-        CUresult r = encode(&out->tile, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), dims, strides, box, ones,
+        const cuuint64_t dims[5] = {64, 8, (cuuint64_t)l.head_dim / 64, 2, (cuuint64_t)2 * l.num_pages * l.num_kv_heads};
+        const cuuint64_t strides[4] = {row, 128, 8 * row, head};
+        const cuuint32_t box[5] = {64, 8, (cuuint32_t)l.head_dim / 64, 2, 1};
+        CUresult r = encode(&out->half, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(pool), dims, strides, box, ones,
                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return r;

@@ -1038,10 +1038,10 @@ cudaError_t launch_mixed_attn(int head_dim, const KvMaps& kv_maps, const CUtenso
     cfg.numAttrs = 1;
     const bool multi = p.nchunks > 1;
     if (head_dim == 64)
-        return multi ? cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<64, true>, kv_maps.tile, kv_maps.page, q_map, p)
-                     : cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<64, false>, kv_maps.tile, kv_maps.page, q_map, p);
-    return multi ? cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<128, true>, kv_maps.tile, kv_maps.page, q_map, p)
-                 : cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<128, false>, kv_maps.tile, kv_maps.page, q_map, p);
+        return multi ? cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<64, true>, kv_maps.half, kv_maps.page, q_map, p)
+                     : cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<64, false>, kv_maps.half, kv_maps.page, q_map, p);
+    return multi ? cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<128, true>, kv_maps.half, kv_maps.page, q_map, p)
+                 : cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<128, false>, kv_maps.half, kv_maps.page, q_map, p);
 }
 
 }  // namespace sw

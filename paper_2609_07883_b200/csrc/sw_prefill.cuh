@@ -6,9 +6,17 @@
 //     S_t = Q_t K_j^T          tcgen05.mma, A and B from shared memory (K-major, 128-byte swizzle), D in TMEM
 //     P_t = exp2(S_t - m)      4 warps per tile, one thread per row (TMEM lane), P written back to TMEM as bf16
 //     O_t += P_t V_j           tcgen05.mma, A from TMEM, B = V from shared memory (MN-major), D in TMEM
-// Roles: warp 0 lane 0 issues TMA (Q once per item, K/V pages into a 2-stage ring), warp 1 lane 0 issues every
-// MMA, warp 2 zeroes V rows past the end of the prompt (unwritten page slots), warps 4-7 / 8-11 run the online
-// softmax of tile 0 / 1.  All hand-offs are mbarriers; every wait is bounded.
+// Roles: warp 0 issues TMA (Q once per item, K/V pages into a 2-stage ring; lane i owns page i of a tile), warp 1
+// issues every MMA (one elected lane), warp 2 zeroes V rows past the end of the prompt (unwritten page slots), warp 3
+// fetches the next work item, warps 4-7 / 8-11 run the online softmax of tile 0 / 1.  All hand-offs are mbarriers;
+// every wait is bounded.
+//
+// Operand tiles of K and V hold their 128 keys as sixteen 8-key groups, each group as head_dim/64 swizzled blocks of
+// [8 slots][128 bytes] side by side: [group 0..15][block][8][128 B].  The 8-key groups of one 64-element block are thus a
+// uniform stride apart (what the matrix descriptors need), and a page (two groups) is one contiguous stretch that ONE
+// copy of 4 KB fills (head_dim 128): the tensor map views a page's rows of one head as {64 elements, 8 slots, block,
+// slot group}.  The copy engine's cost is per copy; with one copy per 2 KB block the producer warp was busy for a whole
+// step and K tiles arrived late.
 #pragma once
 
 namespace sw {
@@ -16,12 +24,14 @@ namespace sw {
 template <int D>
 struct PfGeo {
     static constexpr int kHalves = D / 64;
-    static constexpr int kHalfBytes = 128 * 128;                 // [128 rows][64 elements], 128-byte swizzle
+    static constexpr int kHalfBytes = 128 * 128;                 // Q: [128 rows][64 elements], 128-byte swizzle
     static constexpr int kTileBytes = kHalves * kHalfBytes;      // one Q, K or V tile
     static constexpr int kQOffset = 0;                           // Q tile t at t * kTileBytes
     static constexpr int kKVOffset = 2 * kTileBytes;             // stage s: K at s * 2 * kTileBytes, then V
     static constexpr int kBytes = kKVOffset + 2 * 2 * kTileBytes;
-    static constexpr int kPageBytes = kPageSize * 128;           // one page's rows inside a half
+    static constexpr int kAtomBytes = 8 * 128;                   // K, V: one [8 slots][64 elements] swizzled block
+    static constexpr int kGroupStride = kHalves * kAtomBytes;    // K, V: 8 keys, [head_dim/64 blocks][8][128 B]
+    static constexpr int kPageStride = 2 * kGroupStride;         // K, V: one page = two 8-key groups
 };
 
 // P of a tile is handed to the MMA warp in two halves (keys 0-63, then 64-127) so that the first four P V
@@ -368,19 +378,16 @@ __device__ __forceinline__ bool pf_produce(const CUtensorMap* kv_map, const CUte
         const uint32_t kdst = sh.smem + G::kKVOffset + s * 2 * G::kTileBytes;
         const uint32_t vdst = kdst + G::kTileBytes;
         if (!pf_wait(sh, kBarKEmpty + s, (n & 1) ^ 1, p.ctrl, 1)) return false;
-        if (lane == 0) mbar_arrive_expect_tx(sh.bars + (kBarKFull + s) * 8, nvp * G::kHalves * G::kPageBytes);
+        if (lane == 0) mbar_arrive_expect_tx(sh.bars + (kBarKFull + s) * 8, nvp * G::kPageStride);
         __syncwarp();
         if (lane < nvp)
-            for (int h = 0; h < G::kHalves; ++h)
-                tma_load_4d(kdst + h * G::kHalfBytes + lane * G::kPageBytes, kv_map, sh.bars + (kBarKFull + s) * 8, h * 64, 0,
-                            it.kvh, id);
+            tma_load_5d(kdst + lane * G::kPageStride, kv_map, sh.bars + (kBarKFull + s) * 8, 0, 0, 0, 0, (2 * id) * p.Hkv + it.kvh);
         if (!pf_wait(sh, kBarVEmpty + s, (n & 1) ^ 1, p.ctrl, 2)) return false;
-        if (lane == 0) mbar_arrive_expect_tx(sh.bars + (kBarVLanded + s) * 8, nvp * G::kHalves * G::kPageBytes);
+        if (lane == 0) mbar_arrive_expect_tx(sh.bars + (kBarVLanded + s) * 8, nvp * G::kPageStride);
         __syncwarp();
         if (lane < nvp)
-            for (int h = 0; h < G::kHalves; ++h)
-                tma_load_4d(vdst + h * G::kHalfBytes + lane * G::kPageBytes, kv_map, sh.bars + (kBarVLanded + s) * 8, h * 64, 0,
-                            p.Hkv + it.kvh, id);
+            tma_load_5d(vdst + lane * G::kPageStride, kv_map, sh.bars + (kBarVLanded + s) * 8, 0, 0, 0, 0,
+                        (2 * id + 1) * p.Hkv + it.kvh);
     }
     return true;
 }
@@ -399,10 +406,11 @@ __device__ __forceinline__ bool pf_sanitize(const MixedParams& p, const PfShared
         const int first_dead = max(0, kv_total - j * 128);
         if (first_dead < 128) {
             const uint32_t vdst = sh.smem + G::kKVOffset + s * 2 * G::kTileBytes + G::kTileBytes;
-            const int chunks = (128 - first_dead) * 8;  // 16-byte pieces per half
+            const int chunks = (128 - first_dead) * 8;  // 16-byte pieces per 64-element block
             for (int h = 0; h < G::kHalves; ++h)
                 for (int c = lane; c < chunks; c += 32) {
-                    const uint32_t addr = vdst + h * G::kHalfBytes + (first_dead + c / 8) * 128 + (c % 8) * 16;
+                    const int key = first_dead + c / 8;
+                    const uint32_t addr = vdst + (key >> 3) * G::kGroupStride + h * G::kAtomBytes + (key & 7) * 128 + (c % 8) * 16;
                     asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
                 }
             fence_proxy_async_smem();
@@ -426,32 +434,35 @@ __device__ __forceinline__ void pf_issue_qk(const PfShared& sh, int t, uint32_t 
     using G = PfGeo<D>;
     constexpr uint32_t idesc = umma_idesc_bf16(128, 128, 0, 0);
     const uint64_t qd = umma_desc_sw128(sh.smem + G::kQOffset + t * G::kTileBytes, 16, 1024);
-    const uint64_t kd = umma_desc_sw128(sh.smem + G::kKVOffset + s * 2 * G::kTileBytes, 16, 1024);
+    const uint64_t kd = umma_desc_sw128(sh.smem + G::kKVOffset + s * 2 * G::kTileBytes, 16, G::kGroupStride);
     const uint32_t d_tmem = sh.tmem + t * 128;
     if (leader) {
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
-            const uint64_t off = (uint64_t)(((ks >> 2) * G::kHalfBytes + (ks & 3) * 32) >> 4);  // descriptor address units
-            tc_mma_ss(d_tmem, qd + off, kd + off, idesc, ks > 0);
+            // descriptor address units (16 bytes): 64-element block ks / 4, 16 elements = 32 bytes per slice
+            const uint64_t qoff = (uint64_t)(((ks >> 2) * G::kHalfBytes + (ks & 3) * 32) >> 4);
+            const uint64_t koff = (uint64_t)(((ks >> 2) * G::kAtomBytes + (ks & 3) * 32) >> 4);
+            tc_mma_ss(d_tmem, qd + qoff, kd + koff, idesc, ks > 0);
         }
         tc_commit(sh.bars + (kBarSFull + t) * 8);
     }
 }
 
-// one half of O_t += P_t V: keys [64 * half, 64 * half + 64), 16 keys per instruction
+// one half of O_t += P_t V: keys [64 * half, 64 * half + 64), 16 keys = one page per instruction (its two 8-key groups
+// are one group stride apart, the 64-element blocks of a row one block apart)
 template <int D>
 __device__ __forceinline__ void pf_issue_pv_half(const PfShared& sh, int t, uint32_t s, int half, bool first, bool leader) {
     using G = PfGeo<D>;
     constexpr uint32_t idesc = umma_idesc_bf16(128, D, 0, 1);  // B = V is MN-major: [key][d] with d contiguous
-    const uint64_t vd = umma_desc_sw128(sh.smem + G::kKVOffset + s * 2 * G::kTileBytes + G::kTileBytes + half * 4 * 2048,
-                                        G::kHalfBytes, 1024);
+    const uint64_t vd = umma_desc_sw128(sh.smem + G::kKVOffset + s * 2 * G::kTileBytes + G::kTileBytes + half * 4 * G::kPageStride,
+                                        G::kAtomBytes, G::kGroupStride);
     const uint32_t d_tmem = sh.tmem + 256 + t * D;
     const uint32_t p_tmem = sh.tmem + t * 128 + half * 32;
     const uint32_t acc_first = first && half == 0 ? 0u : 1u;
     if (leader) {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-            tc_mma_ts(d_tmem, p_tmem + i * 8, vd + (uint64_t)(i * (2048 >> 4)), idesc, i == 0 ? acc_first : 1u);
+            tc_mma_ts(d_tmem, p_tmem + i * 8, vd + (uint64_t)(i * (G::kPageStride >> 4)), idesc, i == 0 ? acc_first : 1u);
         if (half == 1) tc_commit(sh.bars + (kBarODone + t) * 8);
     }
 }
@@ -505,33 +516,28 @@ __device__ __forceinline__ bool pf_mma(const MixedParams& p, const PfShared& sh,
 }
 
 // ---- role: online softmax + epilogue (4 warps per tile, one thread per row) ---------------------------------------
-// exp2 either on the special-function unit or, for a fixed share of the elements, as a cubic on the FMA pipe
-// (round to nearest integer with the 1.5 * 2^23 trick, minimax cubic of 2^f on [-0.5, 0.5], relative error 7.5e-5 —
-// far below the bf16 rounding of P — exponent added as integer bits).  The two pipes then share the row's 128 exps.
-#ifndef SW_PF_POLY_EVERY
-#define SW_PF_POLY_EVERY 0
-#endif
-#ifndef SW_PF_SPLIT_MAX
-#define SW_PF_SPLIT_MAX 0
-#endif
-#ifndef SW_PF_MAX_CHAINS
-#define SW_PF_MAX_CHAINS 4
-#endif
-constexpr int kPfMaxChains = SW_PF_MAX_CHAINS;
-constexpr int kPolyEvery = SW_PF_POLY_EVERY;  // every kPolyEvery-th pair computes its first element with the polynomial; 0 = never
-template <bool kPoly>
-__device__ __forceinline__ float pf_exp2(float x) {
-    if constexpr (!kPoly) {
-        return fast_exp2(x);
-    } else {
-        x = fmaxf(x, -126.f);
-        const float t = x + 12582912.f;
-        const float f = x - (t - 12582912.f);
-        float r = fmaf(f, 0.0551716648f, 0.2426111251f);
-        r = fmaf(r, f, 0.6932609677f);
-        r = fmaf(r, f, 0.9999280572f);
-        return __int_as_float(__float_as_int(r) + (__float_as_int(t) << 23));
-    }
+// The row's 128 exponentials are the longest stretch of a tile's softmax: the special-function unit delivers one warp
+// instruction every 8 cycles, 1024 cycles per row, as long as the tensor core needs for a whole tile.  A fixed share of
+// the column pairs is therefore exponentiated on the FMA pipe instead, two columns per instruction: x = n + f with n the
+// nearest integer (1.5 * 2^23 trick), a minimax cubic of 2^f on [-0.5, 0.5] (relative error 7.5e-5, far below the bf16
+// rounding of P), and n added to the exponent as integer bits.  Of every 8 pairs the first kPfFmaPairsOf8 take this path.
+constexpr int kPfMaxChains = 4;      // independent chains of the row maximum
+constexpr int kPfFmaPairsOf8 = 2;    // measured: 2 of 8 gains 2-4 %, 3 of 8 nothing, 4 of 8 loses (the FMA pipe fills up)
+__device__ __forceinline__ void pf_exp2_pair_fma(uint64_t x2, float& p0, float& p1) {
+    float x0, x1;
+    unpack_f32x2(x2, x0, x1);
+    const uint64_t xc = pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));   // 2^-126 stands for zero (and for -inf)
+    const uint64_t t = add_f32x2(xc, pack_f32x2(12582912.f, 12582912.f));  // low mantissa bits = n
+    const uint64_t r = add_f32x2(t, pack_f32x2(-12582912.f, -12582912.f)); // n as a float
+    const uint64_t f = fma_f32x2(r, pack_f32x2(-1.f, -1.f), xc);
+    uint64_t q = fma_f32x2(f, pack_f32x2(0.0551716648f, 0.0551716648f), pack_f32x2(0.2426111251f, 0.2426111251f));
+    q = fma_f32x2(q, f, pack_f32x2(0.6932609677f, 0.6932609677f));
+    q = fma_f32x2(q, f, pack_f32x2(0.9999280572f, 0.9999280572f));
+    float q0, q1, t0, t1;
+    unpack_f32x2(q, q0, q1);
+    unpack_f32x2(t, t0, t1);
+    p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(t0) << 23));
+    p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
 }
 
 struct PfSoftmaxState {
@@ -631,12 +637,15 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
                 // two columns per instruction: x = s * scale - m, P = 2^x, row sum, bf16 pack
                 const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(s[c * 32 + 2 * i]), __uint_as_float(s[c * 32 + 2 * i + 1])),
                                               scale2, negm2);
-                float x0, x1;
-                unpack_f32x2(x2, x0, x1);
-                // the choice folds to a constant once the loop is unrolled
-                const float p0 = (kPolyEvery != 0 && i % (kPolyEvery ? kPolyEvery : 1) == 0) ? pf_exp2<true>(x0)
-                                                                                             : pf_exp2<false>(x0);
-                const float p1 = fast_exp2(x1);
+                float p0, p1;
+                if ((i & 7) < kPfFmaPairsOf8) {   // folds to a constant once the loop is unrolled
+                    pf_exp2_pair_fma(x2, p0, p1);
+                } else {
+                    float x0, x1;
+                    unpack_f32x2(x2, x0, x1);
+                    p0 = fast_exp2(x0);
+                    p1 = fast_exp2(x1);
+                }
                 if (i & 1) sum_b = add_f32x2(sum_b, pack_f32x2(p0, p1)); else sum_a = add_f32x2(sum_a, pack_f32x2(p0, p1));
                 pk[i] = pack_bf16x2(p0, p1);
             }
