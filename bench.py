@@ -35,11 +35,12 @@ ROOT = Path(__file__).resolve().parent
 sys.path.insert(0, str(ROOT))
 
 from paper_2609_07883_b200 import workloads as W  # noqa: E402
+from paper_2609_07883_b200.clocks import ClockSampler  # noqa: E402
 
 NOMINAL_HBM_GBS = 8000.0
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-MIN_WINDOW_MS = 200.0       # every timed window is repeated until it is at least this long
+MIN_WINDOW_MS = 200.0       # every timed window is repeated until it is at least this long (--min-window-ms)
 
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of sw_mixed_attn_kernel (KV append fused in) from ncu captures
 # of exactly these workloads, keyed by (workload, decodes, chunk, prefix, variant); the summary that holds each figure is
@@ -121,69 +122,6 @@ def describe(workload: str, batch: W.MixedBatch) -> str:
     return (f"{workload} iteration, Llama-3-8B attention shape 32/8/128 bf16, 16-token pages: {batch.num_decode} decodes with "
             f"contexts {CONTEXTS[workload]} (total {batch.total_decode_ctx} tokens) + prefill chunk C={batch.chunk_len} at "
             f"prefix {batch.prefix_len}")
-
-
-# ---------------------------------------------------------------------------------------------------------------
-# clocks: one nvidia-smi sampler for the whole run; every timed window picks its own samples by time stamp
-# ---------------------------------------------------------------------------------------------------------------
-class ClockSampler:
-    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-             "clocks_event_reasons.sw_power_cap")
-    REASONS = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-
-    def __init__(self, gpu_index: int, period_ms: int = 50):
-        self.gpu_index, self.period_ms = gpu_index, period_ms
-        self.proc = self.path = None
-        self.rows = None
-
-    def start(self):
-        try:
-            fd, self.path = tempfile.mkstemp(suffix=".csv")
-            os.close(fd)
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", str(self.period_ms)],
-                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
-        except Exception:
-            self.proc = None
-
-    def stop(self):
-        if self.proc is None:
-            self.rows = []
-            return
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        rows = []
-        try:
-            for line in open(self.path).read().splitlines():
-                f = [x.strip() for x in line.split(",")]
-                if len(f) < 8:
-                    continue
-                try:
-                    ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
-                    rows.append((ts, float(f[1]), float(f[2]), float(f[3]),
-                                 [name for name, val in zip(self.REASONS, f[4:8]) if val.lower().startswith("active")]))
-                except ValueError:
-                    continue
-            os.unlink(self.path)
-        except Exception:
-            pass
-        self.rows = rows
-
-    def window(self, t0: float, t1: float) -> dict:
-        """Median SM clock, maximum power and the throttle reasons seen between two host time stamps."""
-        if not self.rows:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"], "samples": 0}
-        rows = [r for r in self.rows if t0 <= r[0] <= t1]
-        if not rows:   # a window shorter than the sampling period: the nearest sample
-            mid = 0.5 * (t0 + t1)
-            rows = [min(self.rows, key=lambda r: abs(r[0] - mid))]
-        reasons = sorted({x for r in rows for x in r[4]})
-        return {"sm_mhz": float(np.median([r[1] for r in rows])), "sm_max_mhz": float(max(r[2] for r in rows)),
-                "power_w_max": float(max(r[3] for r in rows)), "reasons": reasons, "samples": len(rows)}
 
 
 # ---------------------------------------------------------------------------------------------------------------
@@ -474,13 +412,13 @@ def run_ours(args) -> dict:
 
     # (1) the timed region: K steps of the whole iteration, device-timed, repeated until it is 200 ms long
     step = case.stepper(batch)
-    windows["mixed"] = time_window(step, args.steps, MIN_WINDOW_MS, sync_all, reduce_max, args.warmup)
+    windows["mixed"] = time_window(step, args.steps, args.min_window_ms, sync_all, reduce_max, args.warmup)
     B.sw_check_status(case.ctx)
     launches = args.steps * len(windows["mixed"][0])
     # (2) the decode part and the prefill part alone, same pools, same rotation
     for name in ("decode_only", "prefill_only"):
         if name in variants:
-            windows[name] = time_window(case.stepper(variants[name]), args.steps, MIN_WINDOW_MS, sync_all, reduce_max, 3)
+            windows[name] = time_window(case.stepper(variants[name]), args.steps, args.min_window_ms, sync_all, reduce_max, 3)
     B.sw_check_status(case.ctx)
     us = float(np.median(windows["mixed"][0]))
     agg = whole_job(us, world, batch.chunk_len, batch.num_decode, sharded)   # the windows hold the max over ranks already
@@ -524,7 +462,7 @@ def run_ours(args) -> dict:
             w = attention_work(b)
             tw = {}
             for name, vb in variants_of(b).items():
-                per_step, span = time_window(c.stepper(vb), args.steps, MIN_WINDOW_MS, sync_all, reduce_max, 3)
+                per_step, span = time_window(c.stepper(vb), args.steps, args.min_window_ms, sync_all, reduce_max, 3)
                 row[name + "_us"] = spread(per_step)
                 tw[name] = (per_step, span)
             B.sw_check_status(c.ctx)
@@ -628,6 +566,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="time the named workload only")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--min-window-ms", type=float, default=MIN_WINDOW_MS,
+                    help="every timed window repeats its K-step loop until it is this long (0: once; for profiler captures)")
     ap.add_argument("--parallel", default="replicas", choices=["replicas", "heads"],
                     help="N > 1: independent replicas (default) or one iteration sharded by KV heads, no collective either way")
     args = ap.parse_args()

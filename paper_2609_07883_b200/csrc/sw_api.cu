@@ -69,6 +69,7 @@ struct sw_ctx {
     sw_layout layout;
     int device = 0;
     int num_sms = 0;
+    float stage_us = 0.f, step_us = 0.f;  // planning estimates from the device's clocks (sw::device_timing)
     bool grid_resident = false;  // the persistent grid fits the device at once (needed by the fused append + attention launch)
     int max_chunk = 0, max_decode = 0;
     int64_t max_pages = 0;
@@ -230,12 +231,17 @@ sw_status sw_create(const sw_layout* layout, int device, void* workspace, size_t
         }
     } restore{caller_device, device};
     if (caller_device != device) SW_CUDA(cudaSetDevice(device));
+    int mem_khz = 0, bus_bits = 0, sm_khz = 0;
+    SW_CUDA(cudaDeviceGetAttribute(&mem_khz, cudaDevAttrMemoryClockRate, device));
+    SW_CUDA(cudaDeviceGetAttribute(&bus_bits, cudaDevAttrGlobalMemoryBusWidth, device));
+    SW_CUDA(cudaDeviceGetAttribute(&sm_khz, cudaDevAttrClockRate, device));
     sw_ctx* ctx = new (std::nothrow) sw_ctx();
     if (!ctx) return sw_fail(SW_ERR_INVALID_ARG, "sw_create: out of host memory");
     ctx->layout = *layout;
     if (ctx->layout.sm_scale <= 0.f) ctx->layout.sm_scale = 1.0f / std::sqrt((float)layout->head_dim);
     ctx->device = device;
     ctx->num_sms = std::min(prop.multiProcessorCount, sw::kMaxCtas);
+    sw::device_timing(mem_khz, bus_bits, sm_khz, layout->head_dim, &ctx->stage_us, &ctx->step_us);
     ctx->max_chunk = max_chunk;
     ctx->max_decode = max_decode;
     ctx->max_pages = max_pages;
@@ -304,7 +310,7 @@ sw_status sw_kv_append(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const 
     p.v_new = static_cast<const __nv_bfloat16*>(v_new);
     p.pool = static_cast<__nv_bfloat16*>(kv_pool);
     p.ctrl = reinterpret_cast<int32_t*>(ctx->ws + ctx->w.ctrl);
-    SW_CUDA(sw::launch_kv_append(p, static_cast<cudaStream_t>(stream)));
+    SW_CUDA(sw::launch_kv_append(p, ctx->num_sms, static_cast<cudaStream_t>(stream)));
     return SW_OK;
 }
 
@@ -333,6 +339,10 @@ sw_status run_mixed(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const voi
     p.num_pages = l.num_pages;
     p.sm_scale = l.sm_scale;
     p.sm_scale_log2 = l.sm_scale * 1.4426950408889634f;
+    p.stage_us = ctx->stage_us;
+    p.step_us = ctx->step_us;
+    p.stages_per_us = 1.f / ctx->stage_us;
+    p.steps_per_stage = ctx->stage_us / ctx->step_us;
     p.C = ch.rows;
     p.n = batch->num_decode;
     p.nchunks = ch.n;

@@ -34,6 +34,10 @@ struct MixedParams {
     int64_t num_pages;
     float sm_scale;       // softmax scale
     float sm_scale_log2;  // sm_scale * log2(e)
+    // planning estimates, from the device's clocks (device_timing): microseconds in which the whole device streams one
+    // (page, kv head) stage of K and V, and microseconds of one 128-key step of a chunk-prefill entry
+    float stage_us, step_us;
+    float stages_per_us, steps_per_stage;   // 1 / stage_us and stage_us / step_us, worked out on the host
     // batch.  C is the number of chunk rows of the iteration: the rows of its prefill chunks, one chunk after the
     // other.  Chunk j has cC[j] tokens at prefix cP[j], starts at row cRow0[j] and its prompt's page list starts at
     // prefill_pages[cPage0[j]] (cPage0[nchunks] = num_prefill_pages).
@@ -122,7 +126,16 @@ inline CUresult encode_kv_maps(EncodeTiledFn encode, const sw_layout& l, const v
 }
 
 // launchers (sw_kernels.cu)
-cudaError_t launch_kv_append(const AppendParams& p, cudaStream_t stream);
+cudaError_t launch_kv_append(const AppendParams& p, int num_sms, cudaStream_t stream);
+// MixedParams::stage_us / step_us for a device: the memory system streams about 0.76 of clock x bus width x 2 (measured
+// against a plain copy on B200: 6.2 of 8.2 TB/s), and a 128-key step of a chunk-prefill entry takes about 4300 SM
+// cycles while other CTAs stream decode pages (measured; 2.2 us at 1965 MHz).
+inline void device_timing(int mem_clock_khz, int bus_width_bits, int sm_clock_khz, int head_dim, float* stage_us, float* step_us) {
+    const double bytes_per_us = 0.76 * 2.0 * (double)mem_clock_khz * 1e3 * ((double)bus_width_bits / 8.0) / 1e6;
+    const double stage_bytes = 2.0 * kPageSize * head_dim * 2;   // K and V rows of one head in a page
+    *stage_us = (float)(stage_bytes / bytes_per_us);
+    *step_us = (float)(4300.0 / ((double)sm_clock_khz / 1e3));
+}
 cudaError_t launch_mixed_attn(int head_dim, const KvMaps& kv_maps, const CUtensorMap& q_map, const MixedParams& p,
                               int num_sms, cudaStream_t stream);
 cudaError_t configure_kernels(int head_dim);

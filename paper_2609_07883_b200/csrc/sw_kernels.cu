@@ -98,12 +98,12 @@ __global__ void sw_kv_append_kernel(const AppendParams p) {
     append_rows<true>(p, p.D, (int64_t)blockIdx.x * blockDim.x + threadIdx.x, (int64_t)gridDim.x * blockDim.x);
 }
 
-cudaError_t launch_kv_append(const AppendParams& p, cudaStream_t stream) {
+cudaError_t launch_kv_append(const AppendParams& p, int num_sms, cudaStream_t stream) {
     const int64_t total = (int64_t)(p.C + p.n) * (p.Hkv * p.D / 8);
     if (total == 0) return cudaSuccess;
     const int threads = 256;
     int64_t blocks = (total + threads - 1) / threads;
-    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks > (int64_t)num_sms * 8) blocks = (int64_t)num_sms * 8;   // eight 256-thread blocks fill an SM
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)blocks);
     cfg.blockDim = dim3(threads);
@@ -160,25 +160,16 @@ struct Geo {
     static constexpr int kSmemBytes = kMiscOffset + 768;   // 64 ints scan scratch and flags, the plan's counters, the chunk table
 };
 
-#ifndef SW_WIDE_MERGE_SPLITS
-#define SW_WIDE_MERGE_SPLITS 24
-#endif
-constexpr int kWideMergeSplits = SW_WIDE_MERGE_SPLITS;  // from this many units of a request on, its last g units share the merge
+constexpr int kWideMergeSplits = 24;  // from this many units of a request on, its last g units share the merge
 constexpr int kOneRoundMaxPages = 48;  // longest unit (pages) for which one round of units is planned
 constexpr int kPlanCounters = 8;       // shared counters of the plan's block sums, zeroed in the kernel prologue
-// When the CTAs of a single wave of prefill entries turn to decode units: a fixed start-up plus a time per 128-key
-// step of the longest entry (measured with the other CTAs streaming decode pages at the same time), and the rate at
-// which the decode units stream the pool meanwhile.
-#ifndef SW_LATE_STEP_US
-#define SW_LATE_STEP_US 2.2f
-#endif
-constexpr float kLateBaseUs = 1.0f, kLateStepUs = SW_LATE_STEP_US;
-constexpr float kDecodeBytesPerUs = 6.2e6f;
+// When the CTAs of a single wave of prefill entries turn to decode units: a fixed start-up plus the time of the longest
+// entry's 128-key steps (MixedParams::step_us each, with the other CTAs streaming decode pages at the same time); the
+// decode units stream one (page, kv head) stage per MixedParams::stage_us meanwhile.  Both figures come from the
+// device's clocks (see sw_create).
+constexpr float kLateBaseUs = 1.0f;
 constexpr int kMinEarlyCtas = 64;  // CTAs whose rings of page copies keep the memory system busy on their own
-#ifndef SW_MIN_LATE_CTAS
-#define SW_MIN_LATE_CTAS 24
-#endif
-constexpr int kMinLateCtas = SW_MIN_LATE_CTAS;  // fewer late CTAs than this: their delay is not worth units of two sizes
+constexpr int kMinLateCtas = 24;   // fewer late CTAs than this: their delay is not worth units of two sizes
 struct Plan {
     const int* len;     // shared-memory copies of the context lengths and page-list offsets
     const int* indptr;
@@ -866,7 +857,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
         const PfPlan pplan = pf_make_plan<kMulti>(p, base + Geo<D>::kMiscOffset + kChunkTable * 4);
         prefill_ctas = min(pplan.n_entries, (int)gridDim.x);
         late.ctas = prefill_ctas;
-        late.us = kLateBaseUs + kLateStepUs * ((pplan.longest + pplan.pieces - 1) / pplan.pieces);
+        late.us = kLateBaseUs + p.step_us * ((pplan.longest + pplan.pieces - 1) / pplan.pieces);
         const int first_entry = blockIdx.x;
         if (first_entry < pplan.n_entries) {  // CTA-uniform: this CTA has prefill work
             if (warp == 1) {
@@ -896,7 +887,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
 
     const Plan plan = make_plan(p, unit_prefix, reinterpret_cast<int*>(smem + Geo<D>::kLenOffset),
                                 reinterpret_cast<int*>(smem + Geo<D>::kIndptrOffset), scratch, late,
-                                kDecodeBytesPerUs / Geo<D>::kStageBytes);
+                                p.stages_per_us);
     if (plan.total_items > p.max_items) {
         if (threadIdx.x == 0) report(p.ctrl, SW_ERR_WORKSPACE, kSiteScratch, plan.total_items);
     } else {

@@ -95,21 +95,8 @@ __device__ __forceinline__ bool pf_wait(const PfShared& sh, int bar, uint32_t pa
 // CTAs) would leave most SMs idle in the last wave, so each of them is cut along the KV axis into k pieces that run
 // side by side; every piece publishes a partial (m, l, O) and the last piece of an item to arrive merges them.
 // CTAs working at the same time thus stay at similar KV positions (their K/V tiles meet in L2).
-#ifndef SW_PF_MIN_PIECE_STEPS
-#define SW_PF_MIN_PIECE_STEPS 4
-#endif
-constexpr int kPfMinPieceSteps = SW_PF_MIN_PIECE_STEPS;
-#ifndef SW_PF_DECODE_SHARE
-#define SW_PF_DECODE_SHARE 1.0f
-#endif
-constexpr float kPfDecodeShare = SW_PF_DECODE_SHARE;
-// steps of a prefill entry (2.2 us each under decode traffic) that streaming one (page, kv head) stage takes at
-// 6.2 TB/s (8 KB stages of 128-wide heads; an estimate, the same figure serves 64-wide heads)
-constexpr float kPfStepsPerStage = 8192.f / (6.2e6f * 2.2f);
-#ifndef SW_PF_PIECE_COST
-#define SW_PF_PIECE_COST 1
-#endif
-constexpr int kPfPieceCost = SW_PF_PIECE_COST;  // steps' worth of work that cutting an item into one more piece costs
+constexpr int kPfMinPieceSteps = 4;   // never pieces shorter than this many KV steps
+constexpr int kPfPieceCost = 1;       // steps' worth of work that cutting an item into one more piece costs
 
 struct PfPlan {
     int longest, shortest;             // steps of the longest and of the shortest item (items are numbered chunk by chunk)
@@ -261,10 +248,10 @@ __device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p, uint32_t ta
     if (r > 0) plan.pieces = min(G / r, pf_pieces_for(plan.shortest));
     if (plan.pieces > 1 && p.n > 0) {
         // Beside a long decode phase the leftover items need not finish early, and every CTA they occupy is a CTA
-        // that does not stream decode pages meanwhile: pieces about as long as kPfDecodeShare of the decode phase
-        // (all decode pages at the streaming rate, in steps of an entry under decode traffic) are short enough.
-        const float decode_steps = (float)__ldg(p.decode_page_indptr + p.n) * (float)p.Hkv * kPfStepsPerStage;
-        plan.pieces = min(plan.pieces, max(1, (int)ceilf((float)plan.shortest / (kPfDecodeShare * decode_steps))));
+        // that does not stream decode pages meanwhile: pieces about as long as the decode phase (all decode pages at
+        // the streaming rate, counted in steps of an entry under decode traffic) are short enough.
+        const float decode_steps = (float)__ldg(p.decode_page_indptr + p.n) * (float)p.Hkv * p.steps_per_stage;
+        plan.pieces = min(plan.pieces, max(1, (int)ceilf((float)plan.shortest / decode_steps)));
     }
     if (plan.pieces == 1) plan.n_whole = plan.n_items;
     plan.n_entries = plan.n_whole + (plan.n_items - plan.n_whole) * plan.pieces;

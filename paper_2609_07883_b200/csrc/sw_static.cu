@@ -39,6 +39,7 @@ struct DeviceState {
     bool ready = false;
     unsigned char* scratch = nullptr;  // device address of g_static_scratch on this device
     int num_sms = 0;
+    int mem_khz = 0, bus_bits = 0, sm_khz = 0;
     bool configured[2] = {false, false};  // head_dim 64, 128
     EncodeTiledFn encode = nullptr;
 };
@@ -76,6 +77,9 @@ sw_status setup_device(int device, DeviceState** out) {
             return sw_fail(SW_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
         st.scratch = static_cast<unsigned char*>(ptr);
         st.num_sms = prop.multiProcessorCount < sw::kMaxCtas ? prop.multiProcessorCount : sw::kMaxCtas;
+        SW_CUDA(cudaDeviceGetAttribute(&st.mem_khz, cudaDevAttrMemoryClockRate, device));
+        SW_CUDA(cudaDeviceGetAttribute(&st.bus_bits, cudaDevAttrGlobalMemoryBusWidth, device));
+        SW_CUDA(cudaDeviceGetAttribute(&st.sm_khz, cudaDevAttrClockRate, device));
         st.encode = reinterpret_cast<EncodeTiledFn>(fn);
         st.ready = true;
     }
@@ -131,6 +135,9 @@ extern "C" sw_status sw_decode_attn_static(const sw_layout* layout, int device, 
     p.num_pages = l.num_pages;
     p.sm_scale = l.sm_scale > 0.f ? l.sm_scale : 1.0f / std::sqrt((float)l.head_dim);
     p.sm_scale_log2 = p.sm_scale * 1.4426950408889634f;
+    sw::device_timing(st->mem_khz, st->bus_bits, st->sm_khz, l.head_dim, &p.stage_us, &p.step_us);
+    p.stages_per_us = 1.f / p.stage_us;
+    p.steps_per_stage = p.stage_us / p.step_us;
     p.C = 0;
     p.n = batch->num_decode;
     p.decode_kv_len = batch->decode_kv_len;

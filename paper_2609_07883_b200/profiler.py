@@ -35,10 +35,23 @@ def pages_needed(shape: W.AttnShape, n: int, ctx_total: int, prefix: int, chunk:
     return n * (-(-per // S) + 1) + -(-(prefix + chunk) // S) + 8
 
 
+def reps_for(iteration_ns: int, reps: int = 0) -> int:
+    """Timed iterations per grid point: at least 200 below 1 ms per iteration, 100 below 5 ms, 30 otherwise, so that the
+    nearest-rank 99th percentile (the ceil(0.99 * reps)-th smallest sample) leaves out the two / the one largest sample of
+    a short point and is the maximum only for the long ones, where a scheduling hiccup is small beside the iteration.
+    ``reps`` > 0 fixes the number instead."""
+    if reps > 0:
+        return reps
+    return 200 if iteration_ns < 1_000_000 else (100 if iteration_ns < 5_000_000 else 30)
+
+
 def measure_table(ctx, pools, shape: W.AttnShape, num_pages: int, n_grid, ctx_grid, prefix_grid, chunk_grid,
-                  reps: int = 10, warmup: int = 2, seed: int = W.SEED_BASE + 40, progress=None, fused: bool = False) -> dict:
-    """Probe every grid point (``fused``: with the KV append in every launch, as ``sw_mixed_iteration_run`` runs it).  ``ctx`` is a binding.Context big enough for the largest point; ``pools`` the layer
-    stack (list of device tensors).  Returns a plain dict (JSON-serialisable) with P50 and P99 per point."""
+                  reps: int = 0, warmup: int = 3, seed: int = W.SEED_BASE + 40, progress=None, fused: bool = False) -> dict:
+    """Probe every grid point (``fused``: with the KV append in every launch, as ``sw_mixed_iteration_run`` runs it).  ``ctx``
+    is a binding.Context big enough for the largest point; ``pools`` the layer stack (list of device tensors).  Every point
+    gets ``warmup`` untimed iterations (which also size its sample, see ``reps_for``) and then its timed ones.  Returns a
+    plain dict (JSON-serialisable) with the median, the nearest-rank 99th percentile, the maximum and the number of timed
+    iterations of every point."""
     import torch
 
     from . import binding as B
@@ -57,6 +70,10 @@ def measure_table(ctx, pools, shape: W.AttnShape, num_pages: int, n_grid, ctx_gr
     shape4 = (len(n_grid), len(ctx_grid), len(prefix_grid), len(chunk_grid))
     p50 = np.zeros(shape4, dtype=np.int64)
     p99 = np.zeros(shape4, dtype=np.int64)
+    top = np.zeros(shape4, dtype=np.int64)
+    count = np.zeros(shape4, dtype=np.int64)
+    probe = (lambda db, w, r: B.sw_cost_probe_iteration(ctx, pools, db, k_new, v_new, q, out, warmup=w, reps=r)) if fused else (
+        lambda db, w, r: B.sw_cost_probe(ctx, pools, db, q, out, warmup=w, reps=r))
     t0 = time.time()
     for a, n in enumerate(n_grid):
         for b, ctx_total in enumerate(ctx_grid):
@@ -65,21 +82,23 @@ def measure_table(ctx, pools, shape: W.AttnShape, num_pages: int, n_grid, ctx_gr
                     if n == 0 and chunk == 0:
                         continue
                     if chunk == 0 and c_i > 0:      # the decode-only plane does not depend on the prefix
-                        p50[a, b, c_i, e], p99[a, b, c_i, e] = p50[a, b, 0, e], p99[a, b, 0, e]
+                        for plane in (p50, p99, top, count):
+                            plane[a, b, c_i, e] = plane[a, b, 0, e]
                         continue
                     batch = probe_batch(shape, num_pages, int(n), int(ctx_total), int(prefix), int(chunk), rng)
                     db = B.DeviceBatch(batch, dev)
-                    if fused:
-                        m, h, _ = B.sw_cost_probe_iteration(ctx, pools, db, k_new, v_new, q, out, warmup=warmup, reps=reps)
-                    else:
-                        m, h, _ = B.sw_cost_probe(ctx, pools, db, q, out, warmup=warmup, reps=reps)
-                    p50[a, b, c_i, e], p99[a, b, c_i, e] = m, h
+                    first, _, _ = probe(db, warmup, 3)          # a look at the point's duration sizes its sample
+                    r = reps_for(first, reps)
+                    m, h, samples = probe(db, 0, r)
+                    p50[a, b, c_i, e], p99[a, b, c_i, e], top[a, b, c_i, e], count[a, b, c_i, e] = m, h, int(samples.max()), r
         if progress:
             progress(f"n={n}: {time.time() - t0:.1f}s")
     B.sw_check_status(ctx)
     return {"n_grid": [int(x) for x in n_grid], "ctx_grid": [int(x) for x in ctx_grid],
             "prefix_grid": [int(x) for x in prefix_grid], "chunk_grid": [int(x) for x in chunk_grid],
-            "layers": len(pools), "reps": reps, "warmup": warmup, "fused_append": bool(fused), "p50_ns": p50.tolist(), "p99_ns": p99.tolist(),
+            "layers": len(pools), "reps": count.tolist(), "warmup": warmup + 3, "fused_append": bool(fused), "p50_ns": p50.tolist(),
+            "p99_ns": p99.tolist(), "max_ns": top.tolist(),
+            "percentile_rule": "nearest rank: the ceil(0.99 * reps)-th smallest sample (the maximum when reps < 100)",
             "shape": [shape.num_q_heads, shape.num_kv_heads, shape.head_dim, shape.page_size]}
 
 
@@ -99,6 +118,27 @@ def to_cost_table(table: dict, interp: bool = False, which: str = "p99_ns"):
                        np.asarray(table[which], dtype=np.int64), make_monotone=True, interp=interp)
 
 
+def monotone_report(table: dict, cost_table, which: str = "p99_ns") -> dict:
+    """What the library's cumulative maximum did to a measured table: how many grid points it raised, and by how much
+    (the raised value over the measured one), read back from the controller's table at every grid point."""
+    raw = np.asarray(table[which], dtype=np.float64)
+    mono = np.zeros_like(raw)
+    for a, n in enumerate(table["n_grid"]):
+        for b, c in enumerate(table["ctx_grid"]):
+            for d, pre in enumerate(table["prefix_grid"]):
+                for e, k in enumerate(table["chunk_grid"]):
+                    mono[a, b, d, e] = cost_table.lookup(int(n), int(c), int(pre), int(k))
+    live = raw > 0
+    ratio = mono[live] / raw[live]
+    raised = ratio > 1.0
+    p50 = np.asarray(table["p50_ns"], dtype=np.float64)
+    spread = raw[live] / np.maximum(p50[live], 1.0)
+    return {"points": int(live.sum()), "raised": int(raised.sum()), "raised_by_more_than_5_percent": int((ratio > 1.05).sum()),
+            "raised_by_more_than_20_percent": int((ratio > 1.2).sum()),
+            "mean_raise_of_raised": float(ratio[raised].mean()) if raised.any() else 1.0, "max_raise": float(ratio.max()),
+            "p99_over_p50_mean": float(spread.mean()), "p99_over_p50_max": float(spread.max())}
+
+
 # --------------------------------------------------------------------------------------------------------------------
 # cost-surface sweeps of the named workloads (command line)
 # --------------------------------------------------------------------------------------------------------------------
@@ -115,6 +155,23 @@ def _work(batch: W.MixedBatch) -> dict:
             "prefill_flops": 4 * sh.num_q_heads * sh.head_dim * (C * P + C * (C + 1) // 2)}
 
 
+def _timed(ctx, pools, db, q, out, reps: int):
+    """(median, P99) nanoseconds per ITERATION over the layer stack; ``reps`` = 0 sizes the sample by the iteration's length."""
+    from . import binding as B
+
+    first, _, _ = B.sw_cost_probe(ctx, pools, db, q, out, warmup=3, reps=3)
+    p50, p99, _ = B.sw_cost_probe(ctx, pools, db, q, out, warmup=0, reps=reps_for(first, reps))
+    return p50, p99
+
+
+def _with_clocks(rows, spans, sampler):
+    """Attach to every row the clock record of the time window in which it was measured."""
+    sampler.stop()
+    for row, (t0, t1) in zip(rows, spans):
+        row["clocks"] = sampler.window(t0, t1)
+    return rows
+
+
 def sweep(config: str, reps: int, log) -> list:
     """Mixed, prefill-only and decode-only launch times over the workload's (prefix, chunk) grid."""
     import json as _json
@@ -122,6 +179,11 @@ def sweep(config: str, reps: int, log) -> list:
     import torch
 
     from . import binding as B
+    from .clocks import ClockSampler
+
+    sampler = ClockSampler(0)
+    sampler.start()
+    spans = []
 
     peaks_file = Path(__file__).resolve().parent.parent / "MEASURED_PEAKS.json"
     peaks = _json.loads(peaks_file.read_text()) if peaks_file.exists() else {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
@@ -163,13 +225,15 @@ def sweep(config: str, reps: int, log) -> list:
                                                 batch.decode_page_indptr, batch.decode_pages)}
         row = {"prefix": P, "chunk": C, "decodes": n, "decode_ctx": batch.total_decode_ctx, "pool_pages": batch.num_pages}
         w = _work(batch)
+        t_begin = time.time()
         for name, b in variants.items():
             db = B.DeviceBatch(b, dev)
             qq = q if name != "decode_only" else q[C:]
-            p50, p99, _ = B.sw_cost_probe(ctx, pools, db, qq, out[: b.num_rows], warmup=2, reps=reps)
+            p50, p99 = _timed(ctx, pools, db, qq, out[: b.num_rows], reps)
             row[name + "_us_p50"] = p50 / 1e3 / layers
             row[name + "_us_p99"] = p99 / 1e3 / layers
         B.sw_check_status(ctx)
+        spans.append((t_begin, time.time()))
         t_pf, t_dec, t_mix = (row[k + "_us_p50"] * 1e-6 for k in ("prefill_only", "decode_only", "mixed"))
         row["prefill_tflops"] = w["prefill_flops"] / t_pf / 1e12
         row["prefill_frac_measured"] = row["prefill_tflops"] / peaks["bf16_tflops"]
@@ -186,7 +250,7 @@ def sweep(config: str, reps: int, log) -> list:
             f"{row['prefill_frac_nominal']:.2f} of nominal)  decode {row['decode_only_us_p50']:8.1f} us ({row['decode_gbs']:6.0f} GB/s, "
             f"{row['decode_frac_measured']:.2f} / {row['decode_frac_nominal']:.2f})  mixed/(pf+dec) {row['mixed_vs_sum']:.2f}")
         del ctx
-    return rows
+    return _with_clocks(rows, spans, sampler)
 
 
 def sweep_multichunk(reps: int, log) -> list:
@@ -195,7 +259,11 @@ def sweep_multichunk(reps: int, log) -> list:
     import torch
 
     from . import binding as B
+    from .clocks import ClockSampler
 
+    sampler = ClockSampler(0)
+    sampler.start()
+    spans = []
     dev = torch.device("cuda", 0)
     shape = W.LLAMA
     rows = []
@@ -219,8 +287,10 @@ def sweep_multichunk(reps: int, log) -> list:
             ctx = B.Context(shape, batch.num_pages, batch.chunk_len, max(n, 1), pages + 16)
             q = torch.randn(batch.num_rows, shape.num_q_heads, shape.head_dim, device=dev).to(torch.bfloat16)
             out = torch.empty_like(q)
-            p50, p99, _ = B.sw_cost_probe(ctx, pools, B.DeviceBatch(batch, dev), q, out, warmup=2, reps=reps)
+            t_begin = time.time()
+            p50, p99 = _timed(ctx, pools, B.DeviceBatch(batch, dev), q, out, reps)
             B.sw_check_status(ctx)
+            spans.append((t_begin, time.time()))
             flops = 4 * shape.num_q_heads * shape.head_dim * sum(C * P + C * (C + 1) // 2 for P, C in chunks)
             row = {"prefill_tokens": total, "prefix_of_each": prefix, "chunks": k, "decodes": n, "us_p50": p50 / 4e3,
                    "chunk_list": [list(c) for c in chunks],
@@ -230,7 +300,7 @@ def sweep_multichunk(reps: int, log) -> list:
                 f"(p99 {row['us_p99']:.1f}), {flops / 1e9:.1f} GFLOP of prefill")
             del ctx, pools
             torch.cuda.empty_cache()
-    return rows
+    return _with_clocks(rows, spans, sampler)
 
 
 def sweep_few_long_contexts(reps: int, log) -> list:
@@ -239,7 +309,11 @@ def sweep_few_long_contexts(reps: int, log) -> list:
     import torch
 
     from . import binding as B
+    from .clocks import ClockSampler
 
+    sampler = ClockSampler(0)
+    sampler.start()
+    spans = []
     dev = torch.device("cuda", 0)
     shape = W.LLAMA
     rows = []
@@ -254,8 +328,10 @@ def sweep_few_long_contexts(reps: int, log) -> list:
         ctx = B.Context(shape, batch.num_pages, 1, len(lens), int(batch.decode_pages.shape[0]) + 16)
         q = torch.randn(batch.num_rows, shape.num_q_heads, shape.head_dim, device=dev).to(torch.bfloat16)
         out = torch.empty_like(q)
-        p50, p99, _ = B.sw_cost_probe(ctx, pools, B.DeviceBatch(batch, dev), q, out, warmup=3, reps=reps)
+        t_begin = time.time()
+        p50, p99 = _timed(ctx, pools, B.DeviceBatch(batch, dev), q, out, reps)
         B.sw_check_status(ctx)
+        spans.append((t_begin, time.time()))
         kv_bytes = sum(lens) * 2 * shape.num_kv_heads * shape.head_dim * 2
         row = {"contexts": lens, "us_p50": p50 / 2e3, "us_p99": p99 / 2e3, "kv_bytes": kv_bytes,
                "gbs": kv_bytes / (p50 / 2e9) / 1e9}
@@ -263,7 +339,7 @@ def sweep_few_long_contexts(reps: int, log) -> list:
         log(f"contexts {lens}: {row['us_p50']:8.1f} us (p99 {row['us_p99']:.1f}), {kv_bytes / 1e6:.0f} MB of K/V, {row['gbs']:.0f} GB/s")
         del ctx, pools
         torch.cuda.empty_cache()
-    return rows
+    return _with_clocks(rows, spans, sampler)
 
 
 def main(argv=None):
@@ -274,14 +350,15 @@ def main(argv=None):
 
     ap = argparse.ArgumentParser(description="cost surface of a named workload: mixed / prefill-only / decode-only launches")
     ap.add_argument("--config", choices=["chat", "mixed", "long", "multichunk", "longcontext"], default="mixed")
-    ap.add_argument("--reps", type=int, default=10)
+    ap.add_argument("--reps", type=int, default=0,
+                    help="timed iterations per point; 0 = by the point's duration (200 below 1 ms, 100 below 5 ms, else 30)")
     ap.add_argument("--out", default=None)
     args = ap.parse_args(argv)
     build.build()
     if args.config == "multichunk":
         rows = sweep_multichunk(args.reps, lambda s: print(s, flush=True))
     elif args.config == "longcontext":
-        rows = sweep_few_long_contexts(max(args.reps, 20), lambda s: print(s, flush=True))
+        rows = sweep_few_long_contexts(args.reps, lambda s: print(s, flush=True))
     else:
         rows = sweep(args.config, args.reps, lambda s: print(s, flush=True))
     out = args.out or f"cost_surface_{args.config}.json"

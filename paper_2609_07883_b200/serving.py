@@ -133,7 +133,7 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
     nxt, now, done = 0, 0, 0
     iters = chunk_iters = 0
     misses_chunk = misses_decode_only = infeasible_flags = stalled_for_memory = 0
-    chunks, iter_ns, pred_err = [], [], []
+    chunks, iter_ns, pred_err, pred_ratio = [], [], [], []
     fallback_iters = fallback_run = 0
     fallbacks_since_table = reprofiles = 0
     prompts_per_chunk_iter = []
@@ -274,6 +274,7 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
             infeasible_flags += 1
         if predicted and n:
             pred_err.append(dt - predicted)
+            pred_ratio.append(predicted / max(dt, 1))
         if telemetry is not None and n:
             # the table's own prediction, without any margin (several chunks: total tokens at the summed prefix)
             raw = table.lookup(n, total_ctx, sum(r.prefilled for r, _ in admitted) if admitted else 0, c)
@@ -336,6 +337,8 @@ def run_trace(trace: dict, tpot_ms: float, table, execute, shape: W.AttnShape, n
         "tpot_ms_p99_of_request_p99": float(np.percentile(p99_gap, 99)),
         "requests_meeting_tpot": int(np.sum(p99_gap <= tpot_each)),
         "prediction_error_ms_p99": float(np.percentile(pred_err, 99)) / MS if pred_err else 0.0,
+        "predicted_over_measured_mean": float(np.mean(pred_ratio)) if pred_ratio else 0.0,
+        "predicted_over_measured_p50": float(np.median(pred_ratio)) if pred_ratio else 0.0,
         "fallback_iterations": fallback_iters, "reprofiles": reprofiles,
         "mean_prompts_per_chunk_iteration": float(np.mean(prompts_per_chunk_iter)) if prompts_per_chunk_iter else 0.0,
         "margin_ppm": margin_ppm, "c_max": c_max, "quantum": quantum, "wall_s": time.time() - wall0,
@@ -360,7 +363,8 @@ def main(argv=None):
     ap.add_argument("--c-max", type=int, default=4096)
     ap.add_argument("--margin-ppm", type=int, default=50_000)
     ap.add_argument("--table", default=None, help="JSON cost table to reuse; measured first when absent")
-    ap.add_argument("--table-reps", type=int, default=8)
+    ap.add_argument("--table-reps", type=int, default=0,
+                    help="timed iterations per grid point; 0 = by the point's duration (200 below 1 ms, 100 below 5 ms, else 30)")
     ap.add_argument("--max-prefills", type=int, default=1, help="prompts admitted per iteration (first fit when > 1)")
     ap.add_argument("--ttft-slo-ms", type=float, default=None,
                     help="also count the requests that meet both SLOs and the goodput (Sec. 4.3)")
@@ -392,14 +396,16 @@ def main(argv=None):
         ctx_grid = [t for t in (8192, 65536, 196608, 393216) if t < ctx_top] + [ctx_top]
         log(f"measuring cost table: {len(n_grid) * len(ctx_grid) * len(prefix_grid) * len(chunk_grid)} points, {args.layers} layers")
         tab = profiler.measure_table(ctx, pools, shape, args.pages, n_grid, ctx_grid, prefix_grid, chunk_grid,
-                                     reps=args.table_reps, warmup=2, progress=log, fused=True)
+                                     reps=args.table_reps, warmup=3, progress=log, fused=True)
         if args.table:
             profiler.save_table(tab, args.table)
     table = profiler.to_cost_table(tab)
+    stats = profiler.monotone_report(tab, table)
+    log("cost table: " + json.dumps(stats))
     trace = W.bursty_trace(num_requests=args.requests)
     execute = gpu_executor(ctx, pools, shape, args.c_max, max_decode)
     results = {"layers": args.layers, "pages_per_layer": args.pages, "table_points": int(np.prod(np.shape(tab["p99_ns"]))),
-               "runs": []}
+               "table_stats": stats, "runs": []}
     for scale in args.rate_scale:
         scaled = dict(trace, arrival_ns=(trace["arrival_ns"] / scale).astype(np.int64))
         for tpot in args.tpot_ms:
