@@ -46,7 +46,9 @@ MIN_WINDOW_MS = 200.0       # every timed window is repeated until it is at leas
 # of exactly these workloads, keyed by (workload, decodes, chunk, prefix, variant); the summary that holds each figure is
 # named beside it.  A point without a capture reports null.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    ("chat", 64, 512, 512, "mixed"): 311_881_984,     # profiles/sw_mixed_attn_kernel_chat_bench.md
+    ("long", 16, 4096, 98304, "mixed"): 8_196_000_000,        # profiles/dram_traffic_long_bench.md (mean of two launches)
+    ("long", 16, 4096, 98304, "decode_only"): 5_788_000_000,  # profiles/dram_traffic_long_bench.md
+    ("chat", 64, 512, 512, "mixed"): 311_723_520,             # profiles/sw_mixed_attn_kernel_chat_bench.md
 }
 
 
