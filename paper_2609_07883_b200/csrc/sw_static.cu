@@ -94,7 +94,8 @@ extern "C" sw_status sw_decode_attn_static(const sw_layout* layout, int device, 
     if (!layout || !batch) return sw_fail(SW_ERR_INVALID_ARG, "sw_decode_attn_static: null layout or batch");
     const sw_layout& l = *layout;
     if ((l.head_dim != 64 && l.head_dim != 128) || l.page_size != sw::kPageSize || l.num_kv_heads <= 0 ||
-        l.num_q_heads % l.num_kv_heads != 0 || l.num_pages <= 0 || l.num_pages > ((int64_t)1 << 30))
+        l.num_q_heads % l.num_kv_heads != 0 || l.num_pages <= 0 || l.num_pages > ((int64_t)1 << 30) ||
+        2 * l.num_pages * l.num_kv_heads >= ((int64_t)1 << 31))
         return sw_fail(SW_ERR_UNSUPPORTED, "sw_decode_attn_static: unsupported shape");
     const int g = l.num_q_heads / l.num_kv_heads;
     if (!(g == 1 || g == 2 || g == 4 || g == 8)) return sw_fail(SW_ERR_UNSUPPORTED, "sw_decode_attn_static: unsupported head ratio");

@@ -393,7 +393,7 @@ def main(argv=None):
         chunk_grid = [0, 16, 64, 128, 256, 512, 1024, 2048, 4096]
         # the largest context that still leaves room for the longest prompt piece and one ragged page per request
         ctx_top = tokens - (prefix_grid[-1] + chunk_grid[-1]) - shape.page_size * (n_grid[-1] + 64)
-        ctx_grid = [t for t in (8192, 65536, 196608, 393216) if t < ctx_top] + [ctx_top]
+        ctx_grid = [t for t in (8192, 16384, 32768, 65536, 131072, 196608, 393216) if t < ctx_top] + [ctx_top]
         log(f"measuring cost table: {len(n_grid) * len(ctx_grid) * len(prefix_grid) * len(chunk_grid)} points, {args.layers} layers")
         tab = profiler.measure_table(ctx, pools, shape, args.pages, n_grid, ctx_grid, prefix_grid, chunk_grid,
                                      reps=args.table_reps, warmup=3, progress=log, fused=True)
