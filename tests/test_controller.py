@@ -173,7 +173,7 @@ def test_first_fit_over_several_pending_requests_matches_the_oracle(B, oracle):
 
 def test_decode_only_cost_is_read_at_prefix_zero(B, oracle):
     """A table whose c = 0 column differs between prefix points: an iteration without prefill tokens processes no prompt,
-    so both entry points (and the exhaustive scan) judge SW_F_DECODE_INFEASIBLE by the cost at prefix 0, and agree."""
+    so both entry points (and the exhaustive scan) decide SW_F_DECODE_INFEASIBLE by the cost at prefix 0, and agree."""
     grids = ([4], [1000], [0, 100], [0, 16], np.array([10, 20, 50, 60], dtype=np.int64))
     lt, ot = both_tables(B, oracle, *grids)
     one = B.sw_choose_chunk(lt, 0, [30] * 4, 1000, 100, 64)
