@@ -375,13 +375,20 @@ def run_ours(args) -> dict:
     rank, local_rank, world = dist_env()
     if rank == 0:
         build.build()
+    # one rank per GPU; with fewer GPUs than ranks (a single-GPU check of the N > 1 plumbing with --dist-backend gloo) the
+    # ranks share the devices round robin
+    gpu = local_rank % max(1, torch.cuda.device_count())
     if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        if args.dist_backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device("cuda", gpu))
+        else:
+            dist.init_process_group(args.dist_backend)
         dist.barrier()
     from paper_2609_07883_b200 import binding as B
 
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(gpu)
+    dev = torch.device("cuda", gpu)
+    reduce_dev = dev if args.dist_backend == "nccl" else None   # gloo reduces host tensors
     sharded = args.parallel == "heads" and world > 1
     is_default = (args.workload, args.decodes, args.chunk, args.prefix) == ("long",) + WORKLOAD_DEFAULTS["long"][:3]
     do_sweep = world == 1 and not args.no_sweep and is_default
@@ -403,9 +410,9 @@ def run_ours(args) -> dict:
             torch.cuda.synchronize()
 
     def reduce_max(x):
-        return reduce_max_over_ranks(x, dev)
+        return reduce_max_over_ranks(x, reduce_dev)
 
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(gpu)
     if rank == 0:
         sampler.start()
     case = DeviceCase(B, batch, args.layers, dev, W.SEED_BASE + 100 + 1000 * rank, max_chunk=8192 if do_sweep else 0)
@@ -570,6 +577,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--min-window-ms", type=float, default=MIN_WINDOW_MS,
                     help="every timed window repeats its K-step loop until it is this long (0: once; for profiler captures)")
+    ap.add_argument("--dist-backend", default="nccl", choices=["nccl", "gloo"],
+                    help="N > 1: process-group backend (gloo lets several ranks share one GPU to check the plumbing)")
     ap.add_argument("--parallel", default="replicas", choices=["replicas", "heads"],
                     help="N > 1: independent replicas (default) or one iteration sharded by KV heads, no collective either way")
     args = ap.parse_args()
