@@ -52,7 +52,8 @@ typedef struct sw_ctx sw_ctx;               /* opaque; owns tensor-map cache and
 typedef struct sw_cost_table sw_cost_table; /* opaque host object */
 
 /* Attention shape and pool geometry.  Supported: head_dim 64 or 128; page_size 16;
- * num_q_heads / num_kv_heads in {1, 2, 4, 8}. */
+ * num_q_heads / num_kv_heads in {1, 2, 4, 8}; num_pages <= 2^30 and 2 * num_pages * num_kv_heads < 2^31
+ * (the copy engine addresses a page's K or V of one head by a 32-bit block index). */
 typedef struct {
     int32_t num_q_heads, num_kv_heads, head_dim, page_size;
     int64_t num_pages; /* pages in every pool passed to this context */
