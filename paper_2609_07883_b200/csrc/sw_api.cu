@@ -375,7 +375,7 @@ sw_status run_mixed(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const voi
     p.pf_tickets = reinterpret_cast<int32_t*>(ctx->ws + ctx->w.pf_tickets);
     // q as [row][head][element] restricted to the chunk rows: one box = 128 tile rows (token-major, the g heads of a
     // KV head minor) x 64 elements; rows past the chunk read as zero
-    CUtensorMap q_map = kv_maps->half;
+    CUtensorMap q_map = kv_maps->half, out_map = kv_maps->half;
     if (p.C > 0) {
         const cuuint64_t dims[3] = {(cuuint64_t)l.head_dim, (cuuint64_t)l.num_q_heads, (cuuint64_t)p.C};
         const cuuint64_t strides[2] = {(cuuint64_t)l.head_dim * 2, (cuuint64_t)l.num_q_heads * l.head_dim * 2};
@@ -385,8 +385,13 @@ sw_status run_mixed(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const voi
                                  elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return sw_fail(SW_ERR_CUDA, "cuTensorMapEncodeTiled(q) failed with CUresult %d", (int)r);
+        // out has the same shape: tiles whose 128 rows all lie inside a chunk are stored through this map
+        r = ctx->encode(&out_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, out, dims, strides, box, elem_strides,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return sw_fail(SW_ERR_CUDA, "cuTensorMapEncodeTiled(out) failed with CUresult %d", (int)r);
     }
-    SW_CUDA(sw::launch_mixed_attn(l.head_dim, *kv_maps, q_map, p, ctx->num_sms, static_cast<cudaStream_t>(stream)));
+    SW_CUDA(sw::launch_mixed_attn(l.head_dim, *kv_maps, q_map, out_map, p, ctx->num_sms, static_cast<cudaStream_t>(stream)));
     return SW_OK;
 }
 

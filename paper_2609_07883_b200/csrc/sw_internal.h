@@ -136,7 +136,8 @@ inline void device_timing(int mem_clock_khz, int bus_width_bits, int sm_clock_kh
     *stage_us = (float)(stage_bytes / bytes_per_us);
     *step_us = (float)(4300.0 / ((double)sm_clock_khz / 1e3));
 }
-cudaError_t launch_mixed_attn(int head_dim, const KvMaps& kv_maps, const CUtensorMap& q_map, const MixedParams& p,
+cudaError_t launch_mixed_attn(int head_dim, const KvMaps& kv_maps, const CUtensorMap& q_map, const CUtensorMap& out_map,
+                              const MixedParams& p,
                               int num_sms, cudaStream_t stream);
 cudaError_t configure_kernels(int head_dim);
 cudaError_t mixed_attn_resident_ctas_per_sm(int head_dim, int* out);

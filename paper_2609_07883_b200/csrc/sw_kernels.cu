@@ -805,6 +805,7 @@ template <int D, bool kMulti>
 __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid_constant__ CUtensorMap kv_map,
                                                                        const __grid_constant__ CUtensorMap kvp_map,
                                                                     const __grid_constant__ CUtensorMap q_map,
+                                                                    const __grid_constant__ CUtensorMap out_map,
                                                                     const MixedParams p) {
     static_assert(PfGeo<D>::kBytes <= Geo<D>::kRingBytes, "prefill tiles must fit the region shared with the decode ring");
     extern __shared__ uint8_t smem_raw[];
@@ -828,6 +829,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
         for (int i = 0; i < kWarps * kStages; ++i) mbar_init(base + Geo<D>::kBarOffset + i * 8, 1);
         if (tensor_prefill) {
             tma_prefetch_desc(&q_map);
+            tma_prefetch_desc(&out_map);
             pf_init_barriers(base + Geo<D>::kPfBarOffset);
         }
         misc[0] = 0;
@@ -877,7 +879,7 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
             scr.o = p.pf_o;
             scr.tickets = p.pf_tickets;
             scr.flags = &misc[2];
-            prefill_phase<D, kMulti>(&kv_map, &q_map, p, sh, pplan, scr, first_entry, &misc[5]);
+            prefill_phase<D, kMulti>(&kv_map, &q_map, &out_map, p, sh, pplan, scr, first_entry, &misc[5]);
             tc_fence_before_sync();
             __syncthreads();
             if (warp == 1) tmem_dealloc(sh.tmem, 512);
@@ -1015,7 +1017,8 @@ cudaError_t mixed_attn_resident_ctas_per_sm(int head_dim, int* out) {
     return e;
 }
 
-cudaError_t launch_mixed_attn(int head_dim, const KvMaps& kv_maps, const CUtensorMap& q_map, const MixedParams& p,
+cudaError_t launch_mixed_attn(int head_dim, const KvMaps& kv_maps, const CUtensorMap& q_map, const CUtensorMap& out_map,
+                              const MixedParams& p,
                               int num_sms, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)num_sms);
@@ -1029,10 +1032,10 @@ cudaError_t launch_mixed_attn(int head_dim, const KvMaps& kv_maps, const CUtenso
     cfg.numAttrs = 1;
     const bool multi = p.nchunks > 1;
     if (head_dim == 64)
-        return multi ? cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<64, true>, kv_maps.half, kv_maps.page, q_map, p)
-                     : cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<64, false>, kv_maps.half, kv_maps.page, q_map, p);
-    return multi ? cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<128, true>, kv_maps.half, kv_maps.page, q_map, p)
-                 : cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<128, false>, kv_maps.half, kv_maps.page, q_map, p);
+        return multi ? cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<64, true>, kv_maps.half, kv_maps.page, q_map, out_map, p)
+                     : cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<64, false>, kv_maps.half, kv_maps.page, q_map, out_map, p);
+    return multi ? cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<128, true>, kv_maps.half, kv_maps.page, q_map, out_map, p)
+                 : cudaLaunchKernelEx(&cfg, sw_mixed_attn_kernel<128, false>, kv_maps.half, kv_maps.page, q_map, out_map, p);
 }
 
 }  // namespace sw

@@ -543,8 +543,10 @@ struct PfScratch {
 };
 
 template <int D, bool kMulti>
-__device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared& sh, const PfPlan& plan,
-                                           const PfScratch& scr, const PfItem& it, int t, PfSoftmaxState& st) {
+__device__ __forceinline__ bool pf_softmax(const CUtensorMap* out_map, const MixedParams& p, const PfShared& sh,
+                                           const PfPlan& plan, const PfScratch& scr, const PfItem& it, int t,
+                                           PfSoftmaxState& st) {
+    using G = PfGeo<D>;
     if (it.j1 <= it.j0) return true;  // an empty piece (more pieces than steps)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int j_end = min(it.j1, it.nkv[t]);
@@ -669,6 +671,42 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
     if (whole) {
         // epilogue of an item this CTA did alone: O / l -> bf16 -> out
         const float inv = 1.f / l_sum;
+        const int chunk_rows = pf_chunk<D, kMulti>(p, sh, 1, it.chunk);
+        if (it.tok0[t] + 128 / p.group <= chunk_rows) {
+            // Every row of the tile is a row of the chunk: the tile goes to the slot its Q tile came from (the last
+            // Q K^T of the tile has long completed), in the same swizzled layout, and one thread hands it to the copy
+            // engine, which writes whole 128-byte lines instead of 128 threads storing 16 bytes each.
+            const uint32_t stage = sh.smem + G::kQOffset + t * G::kTileBytes + row * 128;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                tmem_ld_32x32b_x32(o_addr + c * 32, v);
+                tc_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int q = c * 4 + i;  // 16-byte piece of the row: half q / 8, position q % 8 (swizzled by the row)
+                    sts_v4(stage + (q >> 3) * G::kHalfBytes + (((q & 7) ^ (row & 7)) << 4),
+                           pack_bf16x2(__uint_as_float(v[8 * i + 0]) * inv, __uint_as_float(v[8 * i + 1]) * inv),
+                           pack_bf16x2(__uint_as_float(v[8 * i + 2]) * inv, __uint_as_float(v[8 * i + 3]) * inv),
+                           pack_bf16x2(__uint_as_float(v[8 * i + 4]) * inv, __uint_as_float(v[8 * i + 5]) * inv),
+                           pack_bf16x2(__uint_as_float(v[8 * i + 6]) * inv, __uint_as_float(v[8 * i + 7]) * inv));
+                }
+            }
+            if (p.lse) p.lse[out_row * p.Hq + head] = (m_ref + __log2f(l_sum)) * 0.6931471805599453f;
+            tc_fence_before_sync();
+            fence_proxy_async_smem();
+            named_barrier_sync(2 + t, 128);
+            if ((warp & 3) == 0 && lane == 0) {
+                const int row0 = pf_chunk<D, kMulti>(p, sh, 2, it.chunk) + it.tok0[t];
+#pragma unroll
+                for (int h = 0; h < G::kHalves; ++h)
+                    tma_store_3d(out_map, sh.smem + G::kQOffset + t * G::kTileBytes + h * G::kHalfBytes, h * 64,
+                                 it.kvh * p.group, row0);
+                tma_store_commit();
+                // the slot is read before this thread reaches the barrier that lets the producer refill it
+                tma_store_wait_read();
+            }
+            return true;
+        }
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {
             tmem_ld_32x32b_x32(o_addr + c * 32, v);
@@ -778,9 +816,9 @@ __device__ __forceinline__ bool pf_softmax(const MixedParams& p, const PfShared&
 // `next` points at two shared-memory ints: the idle warp fetches the following entry from the global counter while
 // the current one is processed and leaves it in next[iteration parity]; everyone reads it after the piece barrier.
 template <int D, bool kMulti>
-__device__ __forceinline__ void prefill_phase(const CUtensorMap* kv_map, const CUtensorMap* q_map, const MixedParams& p,
-                                              const PfShared& sh, const PfPlan& plan, const PfScratch& scr, int first_entry,
-                                              volatile int* next) {
+__device__ __forceinline__ void prefill_phase(const CUtensorMap* kv_map, const CUtensorMap* q_map, const CUtensorMap* out_map,
+                                              const MixedParams& p, const PfShared& sh, const PfPlan& plan,
+                                              const PfScratch& scr, int first_entry, volatile int* next) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint32_t prod_kv_it = 0, san_kv_it = 0;
     PfMmaState mma_state;
@@ -820,10 +858,11 @@ __device__ __forceinline__ void prefill_phase(const CUtensorMap* kv_map, const C
         int entry = first_entry;
         for (int iter = 0; entry < plan.n_entries; ++iter) {
             const PfItem it = pf_entry<kMulti>(p, plan, entry);
-            pf_softmax<D, kMulti>(p, sh, plan, scr, it, (warp - 4) >> 2, sm_state);
+            pf_softmax<D, kMulti>(out_map, p, sh, plan, scr, it, (warp - 4) >> 2, sm_state);
             if (!piece_sync()) break;
             entry = next[iter & 1];
         }
+        tma_store_wait_all();  // the tiles handed to the copy engine are in global memory before the CTA moves on
         setmaxnreg_dec<kPfRegsLaunch>();
     }
 }

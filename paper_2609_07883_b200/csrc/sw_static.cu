@@ -154,6 +154,6 @@ extern "C" sw_status sw_decode_attn_static(const sw_layout* layout, int device, 
     p.part_o = reinterpret_cast<float*>(st->scratch + kOffPartO);
     p.max_items = kStaticMaxItems;
     p.target_items = kStaticTargetItems;
-    SW_CUDA(sw::launch_mixed_attn(l.head_dim, kv_maps, kv_maps.half, p, st->num_sms, s));
+    SW_CUDA(sw::launch_mixed_attn(l.head_dim, kv_maps, kv_maps.half, kv_maps.half, p, st->num_sms, s));
     return SW_OK;
 }
