@@ -19,7 +19,9 @@
  *     sw_mixed_iteration_run, sw_mixed_iteration_host, the cost probes) require that device to be the caller's
  *     current CUDA device and return SW_ERR_INVALID_ARG otherwise; no call changes the current device
  *     (sw_create sets `device` for its own set-up and restores the caller's).
- *   - bf16 tensors are dense, row-major, innermost index last.
+ *   - bf16 tensors are dense, row-major, innermost index last.  The pool, q, k_new, v_new and out must start
+ *     on a 16-byte boundary (the copy engine reads and writes them through tensor maps); a call given a
+ *     pointer that does not returns SW_ERR_INVALID_ARG and launches nothing.
  *   - KV pool layout (elements, bf16):  [num_pages][2 (0 = K, 1 = V)][num_kv_heads][page_size][head_dim].
  *     The pool must hold finite values everywhere a page list can reach (initialise it with zeros): the
  *     unwritten slots of a partly filled last page are read and multiplied by a zero weight.

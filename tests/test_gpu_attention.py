@@ -285,6 +285,16 @@ def test_host_argument_errors(gpu):
     with pytest.raises(B.SwError) as e:
         B.sw_mixed_attn_run(r.ctx, r.pool, B.DeviceBatch(big, r.dev), r.q, r.out)
     assert e.value.status == B.SW_ERR_WORKSPACE
+    # q and out are read and written through tensor maps: a pointer off the 16-byte grid is refused, nothing is launched
+    import torch
+
+    wide = torch.zeros(r.out.numel() + 8, dtype=r.out.dtype, device=r.out.device)
+    skewed = wide[1:1 + r.out.numel()].view(r.out.shape)   # 2 bytes past an aligned address
+    for q, out in ((r.q, skewed), (skewed, r.out)):
+        with pytest.raises(B.SwError) as e:
+            B.sw_mixed_attn_run(r.ctx, r.pool, r.dbatch, q, out)
+        assert e.value.status == B.SW_ERR_INVALID_ARG and "16-byte aligned" in str(e.value)
+    assert B.sw_check_status(r.ctx, raise_on_error=False) == (0, 0)
 
 
 def test_host_buffer_iteration_matches_device_path(gpu, oracle):
