@@ -23,6 +23,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // Offsets of the regions inside the caller's workspace.
 struct WsLayout {
     size_t ctrl, tickets, part_ml, part_o, pf_tickets, pf_ml, pf_o, st_q, st_k, st_v, st_out, st_lse, st_pages, total;
+    int pf_slots;
     int max_items;
 };
 
@@ -51,8 +52,11 @@ WsLayout ws_layout(const sw_layout& l, int max_chunk, int max_decode, int64_t ma
     // 256-row groups of the chunks of one iteration: every chunk may end in a ragged group
     const size_t groups = ((size_t)max_chunk + (256 / g) - 1) / (256 / g) + sw::kMaxChunks;
     w.pf_tickets = off; off = align_up(off + std::max<size_t>(1, groups) * l.num_kv_heads * 2 * 4, 256);
-    w.pf_ml = off;    off = align_up(off + (size_t)sw::kMaxCtas * 2 * 256 * 4, 256);
-    w.pf_o = off;     off = align_up(off + (max_chunk > 0 ? (size_t)sw::kMaxCtas * 2 * 128 * l.head_dim * 4 : 0), 256);
+    // pieces of items publish partial results: one slot per CTA, more where a chunk can hold a whole round of items
+    // (its leftover items may then be cut into pieces that run in several rounds)
+    w.pf_slots = groups * l.num_kv_heads >= 64 ? sw::kPfRoundSlots : sw::kMaxCtas;
+    w.pf_ml = off;    off = align_up(off + (size_t)w.pf_slots * 2 * 256 * 4, 256);
+    w.pf_o = off;     off = align_up(off + (max_chunk > 0 ? (size_t)w.pf_slots * 2 * 128 * l.head_dim * 4 : 0), 256);
     w.st_q = off;     off = align_up(off + rows * l.num_q_heads * l.head_dim * 2, 256);
     w.st_k = off;     off = align_up(off + rows * l.num_kv_heads * l.head_dim * 2, 256);
     w.st_v = off;     off = align_up(off + rows * l.num_kv_heads * l.head_dim * 2, 256);
@@ -372,6 +376,7 @@ sw_status run_mixed(sw_ctx* ctx, void* kv_pool, const sw_batch* batch, const voi
     p.target_items = sw::kTargetItems;
     p.pf_ml = reinterpret_cast<float*>(ctx->ws + ctx->w.pf_ml);
     p.pf_o = reinterpret_cast<float*>(ctx->ws + ctx->w.pf_o);
+    p.pf_slots = ctx->w.pf_slots;
     p.pf_tickets = reinterpret_cast<int32_t*>(ctx->ws + ctx->w.pf_tickets);
     // q as [row][head][element] restricted to the chunk rows: one box = 128 tile rows (token-major, the g heads of a
     // KV head minor) x 64 elements; rows past the chunk read as zero

@@ -17,6 +17,7 @@ constexpr int kTargetItems = 4096;      // split-KV units aimed at per launch (b
 constexpr int kMinSplitTokens = 128;    // never split a decode context finer than this
 constexpr int kMaxGroup = 8;            // query heads per KV head
 constexpr int kMaxCtas = 192;           // persistent CTAs (one per SM) the scratch is sized for
+constexpr int kPfRoundSlots = 3 * kMaxCtas;  // partial results of chunk-prefill pieces that run in several rounds
 constexpr int kMaxChunks = 8;           // prefill chunks (of different prompts) in one iteration
 constexpr int kMaxChunk = 65536;        // chunk tokens per iteration (256-row groups are planned in shared memory)
 
@@ -66,8 +67,9 @@ struct MixedParams {
     int max_items;      // partial-result slots available
     int target_items;   // split-KV units aimed at (<= max_items - n*Hkv)
     // scratch of prefill items finished by several CTAs
-    float* pf_ml;        // [kMaxCtas][2][2][128]
-    float* pf_o;         // [kMaxCtas][2][D / 4][128][4]
+    float* pf_ml;        // [pf_slots][2][2][128]
+    float* pf_o;         // [pf_slots][2][D / 4][128][4]
+    int pf_slots;        // kMaxCtas, or kPfRoundSlots where a chunk can hold a whole round of items
     int32_t* pf_tickets; // [items][2]
 };
 

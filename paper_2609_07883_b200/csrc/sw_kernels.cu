@@ -857,11 +857,13 @@ __global__ void __launch_bounds__(kThreads, 1) sw_mixed_attn_kernel(const __grid
     LateJoin late{0, 0.f};
     if (tensor_prefill) {
         const PfPlan pplan = pf_make_plan<kMulti>(p, base + Geo<D>::kMiscOffset + kChunkTable * 4);
-        prefill_ctas = min(pplan.n_entries, (int)gridDim.x);
+        prefill_ctas = min(pplan.n_entries, pplan.ctas);
         late.ctas = prefill_ctas;
         late.us = kLateBaseUs + p.step_us * ((pplan.longest + pplan.pieces - 1) / pplan.pieces);
+        if (pplan.n_items >= pplan.ctas)  // whole rounds: the prefill CTAs share all items' steps
+            late.us = kLateBaseUs + p.step_us * (0.5f * (float)(pplan.longest + pplan.shortest) * (float)pplan.n_items / (float)pplan.ctas);
         const int first_entry = blockIdx.x;
-        if (first_entry < pplan.n_entries) {  // CTA-uniform: this CTA has prefill work
+        if (first_entry < prefill_ctas) {  // CTA-uniform: this CTA has prefill work
             if (warp == 1) {
                 tmem_alloc(smem_u32(const_cast<int*>(&misc[0])), 512);
                 tmem_relinquish();

@@ -99,6 +99,15 @@ __device__ __forceinline__ bool pf_wait(const PfShared& sh, int bar, uint32_t pa
 // CTAs working at the same time thus stay at similar KV positions (their K/V tiles meet in L2).
 constexpr int kPfMinPieceSteps = 4;   // never pieces shorter than this many KV steps
 constexpr int kPfPieceCost = 1;       // steps' worth of work that cutting an item into one more piece costs
+// Whole rounds of items beside decode requests: the decode pages need the memory system, not the SMs, and about
+// kDecodeCtasAtFullRate CTAs' rings of page copies already draw the full rate.  So a few CTAs take no chunk-prefill work
+// at all and stream decode pages from the start, as many as it takes for the two kinds of work to end together; the
+// leftover items of the others' last round are cut into pieces that may run in several rounds.
+constexpr int kDecodeCtasAtFullRate = 64;
+constexpr float kDecodeCtasMinGain = 0.20f;
+constexpr float kDecodeCtasMinSteps = 48.f;
+constexpr int kPfMinRoundPieceSteps = 24;  // pieces that run in several rounds: at least this many KV steps each
+constexpr int kPfMaxRoundPieces = 12;
 
 struct PfPlan {
     int longest, shortest;             // steps of the longest and of the shortest item (items are numbered chunk by chunk)
@@ -106,6 +115,7 @@ struct PfPlan {
     int n_whole;        // entries [0, n_whole) are whole items
     int pieces;         // k: pieces per tail item (1 = tail items are whole too); several chunks: of the first chunk's
     int n_entries;      // n_whole + (n_items - n_whole) * k; several chunks: every chunk's tail items times its own k
+    int ctas;           // CTAs that take entries (the first ones by index); the others start with decode units
     uint32_t table;     // several chunks: shared address of the chunk table (k of chunk j is field 4)
 };
 
@@ -232,9 +242,10 @@ __device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p, uint32_t ta
         plan.longest = lds_s32(tot + 12);
         plan.shortest = lds_s32(tot + 16);
         plan.pieces = lds_s32(tot + 20);
+        plan.ctas = (int)gridDim.x;
         return plan;
     }
-    const int G = (int)gridDim.x;
+    int G = (int)gridDim.x;
     const int n_tp = pf_num_groups(p.group, p.cC[0]);
     plan.n_items = n_tp * p.Hkv;
     plan.longest = 0;
@@ -243,16 +254,45 @@ __device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p, uint32_t ta
         plan.longest = pf_steps_of_rank(p.group, p.cP[0], p.cC[0], n_tp, 0);
         plan.shortest = pf_steps_of_rank(p.group, p.cP[0], p.cC[0], n_tp, n_tp - 1);
     }
+    bool rounds = false;
+    float decode_steps = 0.f;  // the decode phase at the full streaming rate, in steps of an entry
+    if (p.n > 0) decode_steps = (float)__ldg(p.decode_page_indptr + p.n) * (float)p.Hkv * p.steps_per_stage;
+    if (p.n > 0 && plan.n_items >= G) {  // at least one whole round of items beside decode requests
+        // work in CTA-steps: the items (their lengths fall linearly with the rank) and the decode pages, at the rate of
+        // one CTA and with every CTA drawing 1 / G of the full rate
+        const float wp = 0.5f * (float)(plan.longest + plan.shortest) * (float)plan.n_items;
+        const float wd = decode_steps * (float)kDecodeCtasAtFullRate, wd_all = decode_steps * (float)G;
+        // CTA time the launch saves when few CTAs stream.  Entries run slower while pages are streamed beside them, so
+        // below a fifth of the launch the plain order (every CTA turns to the decode units after its entries) is kept;
+        // it is also kept beside a decode phase so short that latency, not the streaming rate, bounds it.
+        rounds = decode_steps >= kDecodeCtasMinSteps && wd_all - wd >= kDecodeCtasMinGain * (wp + wd_all);
+        // d CTAs streaming for the whole launch finish with the others when d / G is the decode share of the work
+        if (rounds) G -= min(kDecodeCtasAtFullRate, (int)(wd * (float)G / (wp + wd) + 0.5f));
+    }
+    plan.ctas = G;
     const int r = plan.n_items % G;
     plan.n_whole = plan.n_items - r;
     plan.pieces = 1;
-    // the tail items are short ones; size the pieces by the shortest item, never more pieces than fit side by side
-    if (r > 0) plan.pieces = min(G / r, pf_pieces_for(plan.shortest));
-    if (plan.pieces > 1 && p.n > 0) {
+    if (rounds && r > 0) {
+        // The leftover items may run in several rounds of pieces: the k that ends the last round soonest (a piece costs
+        // its steps plus its share of the merge), among those whose partial results fit the scratch.
+        const int kmax = min(min(kPfMaxRoundPieces, p.pf_slots / r), max(1, plan.shortest / kPfMinRoundPieceSteps));
+        int best = 0x7fffffff;
+        for (int k = 1; k <= kmax; ++k) {
+            const int t = ((r * k + G - 1) / G) * ((plan.shortest + k - 1) / k + (k > 1 ? 2 + k / 2 : 0));
+            if (t < best) {
+                best = t;
+                plan.pieces = k;
+            }
+        }
+    } else if (r > 0) {
+        // the tail items are short ones; size the pieces by the shortest item, never more pieces than fit side by side
+        plan.pieces = min(G / r, pf_pieces_for(plan.shortest));
+    }
+    if (!rounds && plan.pieces > 1 && p.n > 0) {
         // Beside a long decode phase the leftover items need not finish early, and every CTA they occupy is a CTA
         // that does not stream decode pages meanwhile: pieces about as long as the decode phase (all decode pages at
         // the streaming rate, counted in steps of an entry under decode traffic) are short enough.
-        const float decode_steps = (float)__ldg(p.decode_page_indptr + p.n) * (float)p.Hkv * p.steps_per_stage;
         plan.pieces = min(plan.pieces, max(1, (int)ceilf((float)plan.shortest / decode_steps)));
     }
     if (plan.pieces == 1) plan.n_whole = plan.n_items;
@@ -846,8 +886,8 @@ __device__ __forceinline__ void prefill_phase(const CUtensorMap* kv_map, const C
             } else if (warp == 2) {
                 if (it.j1 > it.j0) pf_sanitize<D, kMulti>(p, sh, it, san_kv_it);
             } else {
-                // entries 0 .. gridDim.x-1 are the CTAs' first ones; the counter hands out the rest
-                if (lane == 0) next[iter & 1] = (int)gridDim.x + atomicAdd(&p.ctrl[kCtrPrefill], 1);
+                // entries 0 .. plan.ctas-1 are the CTAs' first ones; the counter hands out the rest
+                if (lane == 0) next[iter & 1] = plan.ctas + atomicAdd(&p.ctrl[kCtrPrefill], 1);
             }
             if (!piece_sync()) break;
             entry = next[iter & 1];

@@ -89,6 +89,27 @@ def test_long_context_workload_large_chunks(gpu, oracle):
     run_case(gpu, oracle, half, edge_pairs(gpu, half, np.random.default_rng(8), 4), 106, "long n=16 C=4096 P=98304")
 
 
+@pytest.mark.parametrize("C,P,n,L,fused", [
+    (4096, 4096, 128, 3200, True),      # whole items only, about 30 CTAs stream decode pages from the start
+    (2048, 8192, 96, 4000, False),      # leftover items cut in two, side by side
+    (2048, 12288, 35, 20000, True),     # about 60 leftover items cut in three: 180 pieces for the 98 CTAs that take them
+    (2048, 16384, 47, 20000, False),    # about 60 leftover items cut in three to five, for 97 CTAs
+], ids=["whole_items", "two_pieces", "pieces_in_rounds", "more_pieces_in_rounds"])
+def test_whole_rounds_of_items_beside_many_decode_pages(gpu, oracle, C, P, n, L, fused):
+    """A chunk of at least one whole round of work items (one per SM) beside decode requests whose pages are a tenth of
+    the launch or more: some CTAs take no chunk-prefill entry and stream decode pages from the start, the others share
+    the items, and the items left over after their whole rounds are cut along the KV axis into pieces that may
+    outnumber those CTAs (they are pulled from the counter over several rounds and merged by the last to arrive).
+    The comments give what the plan does on a device of 148 SMs."""
+    rng = np.random.default_rng(50 + C + P)
+    lens = [L - (i * 37) % (L // 4) for i in range(n)]
+    need = sum(-(-x // 16) for x in lens) + (P + C) // 16 + 64
+    batch = W.make_batch(W.LLAMA, need, lens, P, C, rng)
+    rows = gpu.boundary_rows(C, batch.shape.group) + list(range(0, 512, 7))   # the leftover items are the chunk's first rows
+    pairs = sample_pairs(batch, np.random.default_rng(9), sorted(set(rows)), 12)
+    run_case(gpu, oracle, batch, pairs, 150 + n, f"C={C} P={P} beside {n} decodes of up to {L} tokens", fused=fused)
+
+
 def test_page_ids_above_two_to_the_twenty(gpu, oracle):
     """A 70 GB pool (1.1 M pages of 64 KB) with the live pages scattered over all of it: byte offsets pass 2^36."""
     import torch
