@@ -267,7 +267,7 @@ __device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p, uint32_t ta
         // it is also kept beside a decode phase so short that latency, not the streaming rate, bounds it.
         rounds = decode_steps >= kDecodeCtasMinSteps && wd_all - wd >= kDecodeCtasMinGain * (wp + wd_all);
         // d CTAs streaming for the whole launch finish with the others when d / G is the decode share of the work
-        if (rounds) G -= min(kDecodeCtasAtFullRate, (int)(wd * (float)G / (wp + wd) + 0.5f));
+        if (rounds) G -= min(min(kDecodeCtasAtFullRate, G / 2), (int)(wd * (float)G / (wp + wd) + 0.5f));
     }
     plan.ctas = G;
     const int r = plan.n_items % G;
@@ -293,7 +293,23 @@ __device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p, uint32_t ta
         // Beside a long decode phase the leftover items need not finish early, and every CTA they occupy is a CTA
         // that does not stream decode pages meanwhile: pieces about as long as the decode phase (all decode pages at
         // the streaming rate, counted in steps of an entry under decode traffic) are short enough.
-        plan.pieces = min(plan.pieces, max(1, (int)ceilf((float)plan.shortest / decode_steps)));
+        const int kmax = plan.pieces;
+        plan.pieces = min(kmax, max(1, (int)ceilf((float)plan.shortest / decode_steps)));
+        if (plan.n_whole == 0 && decode_steps >= kDecodeCtasMinSteps) {
+            // Fewer items than CTAs beside a decode phase bound by the streaming rate: the CTAs without an entry stream
+            // at (their number / kDecodeCtasAtFullRate) of the full rate while the pieces run, everybody streams what is
+            // left afterwards; the k that ends the launch soonest.
+            float best = 3.0e38f;
+            for (int k = 1; k <= kmax; ++k) {
+                const float t = (float)((plan.shortest + k - 1) / k + (k > 1 ? 2 + k / 2 : 0));
+                const float rate = fminf(1.f, (float)(G - r * k) / (float)kDecodeCtasAtFullRate);
+                const float end = t + fmaxf(0.f, decode_steps - t * rate);
+                if (end < best) {
+                    best = end;
+                    plan.pieces = k;
+                }
+            }
+        }
     }
     if (plan.pieces == 1) plan.n_whole = plan.n_items;
     plan.n_entries = plan.n_whole + (plan.n_items - plan.n_whole) * plan.pieces;
