@@ -50,6 +50,15 @@ def test_mixed_workload_cost_surface_point(gpu, oracle):
     run_case(gpu, oracle, batch, pairs, 102, "mixed n=128 C=1024 P=4096")
 
 
+@pytest.mark.parametrize("C,P", [(256, 28672), (512, 16384), (64, 28672)])
+def test_fewer_items_than_sms_beside_many_decode_pages(gpu, oracle, C, P):
+    """32, 64 or 8 work items of 130 to 225 KV tiles beside the 128 log-normal decodes (1.4 GB of pages): the number of
+    pieces per item is the one that ends the launch soonest when the SMs without a piece stream decode pages meanwhile."""
+    batch = W.mixed_batch(C, P, n=128, rng=W.rng_for(2))
+    pairs = sample_pairs(batch, np.random.default_rng(12), gpu.boundary_rows(C, batch.shape.group), 16)
+    run_case(gpu, oracle, batch, pairs, 160 + C, f"mixed n=128 C={C} P={P}", fused=True)
+
+
 def test_long_context_workload(gpu, oracle):
     rng = W.rng_for(3)
     batch = W.long_batch(1024, 98304, n=16, rng=rng)
