@@ -159,7 +159,24 @@ __device__ __forceinline__ int pf_pieces_for(int steps) {
     return max(1, min(k, steps / kPfMinPieceSteps));
 }
 
-// Several chunks in one iteration: the tail items (the last n_items mod gridDim ones) belong to chunks of very
+// CTAs that take chunk-prefill entries when n_items items of wp steps in all run beside the decode requests (the
+// others start with decode units); G when the plain order is kept.
+__device__ __forceinline__ int pf_entry_ctas(const MixedParams& p, int G, int n_items, float wp, float decode_steps) {
+    if (p.n <= 0 || n_items < G) return G;  // no decode requests, or not even one whole round of items
+    // work in CTA-steps: the decode pages at the rate of one CTA, and with every CTA drawing 1 / G of the full rate
+    const float wd = decode_steps * (float)kDecodeCtasAtFullRate, wd_all = decode_steps * (float)G;
+    // CTA time the launch saves when few CTAs stream.  Entries run slower while pages are streamed beside them, so
+    // below a fifth of the launch the plain order (every CTA turns to the decode units after its entries) is kept;
+    // it is also kept beside a decode phase so short that latency, not the streaming rate, bounds it.
+    if (decode_steps < kDecodeCtasMinSteps || wd_all - wd < kDecodeCtasMinGain * (wp + wd_all)) return G;
+    // d CTAs streaming for the whole launch finish with the others when d / G is the decode share of the work
+    return G - min(min(kDecodeCtasAtFullRate, G / 2), (int)(wd * (float)G / (wp + wd) + 0.5f));
+}
+__device__ __forceinline__ float pf_decode_steps(const MixedParams& p) {  // the decode phase at the full rate, in steps
+    return p.n > 0 ? (float)__ldg(p.decode_page_indptr + p.n) * (float)p.Hkv * p.steps_per_stage : 0.f;
+}
+
+// Several chunks in one iteration: the tail items (the last n_items mod G ones, G the CTAs that take entries) belong to chunks of very
 // different lengths, e.g. the end of a long prompt next to the start of a new one.  Each chunk gets its own piece
 // count, sized by its shortest item; while the tail entries outnumber the CTAs, the chunk with the shortest pieces
 // gives one up.  Run by one whole warp in the kernel prologue, lane j owning chunk j; fills the chunk table:
@@ -167,7 +184,6 @@ __device__ __forceinline__ int pf_pieces_for(int steps) {
 // tail items (fields 5 and 6 hold INT_MAX where nothing may match), then the plan's totals.
 __device__ __forceinline__ void pf_fill_chunk_table(const MixedParams& p, int* tbl) {
     const int lane = threadIdx.x & 31;
-    const int G = (int)gridDim.x;
     int P = 0, C = 0, row0 = 0, page0 = 0;
 #pragma unroll
     for (int j = 0; j < kMaxChunks; ++j)
@@ -190,13 +206,16 @@ __device__ __forceinline__ void pf_fill_chunk_table(const MixedParams& p, int* t
     const int incl = scan(cnt);
     const int before = incl - cnt;
     const int n_items = __shfl_sync(0xffffffffu, incl, kMaxChunks - 1);
-    const int n_whole = n_items - n_items % G;
-    const int tail = max(0, before + cnt - max(before, n_whole));
     int longest = 0, shortest = 0x7fffffff;
     if (n_tp > 0) {
         longest = pf_steps_of_rank(p.group, P, C, n_tp, 0);
         shortest = pf_steps_of_rank(p.group, P, C, n_tp, n_tp - 1);
     }
+    // beside enough decode pages a few CTAs take no entry (the rule of the single-chunk plan; pieces in one round here)
+    const int steps2 = __reduce_add_sync(0xffffffffu, n_tp > 0 ? (longest + shortest) * cnt : 0);
+    const int G = pf_entry_ctas(p, (int)gridDim.x, n_items, 0.5f * (float)steps2, pf_decode_steps(p));
+    const int n_whole = n_items - n_items % G;
+    const int tail = max(0, before + cnt - max(before, n_whole));
     int k = tail > 0 ? pf_pieces_for(shortest) : 1;
     int total = __reduce_add_sync(0xffffffffu, tail * k);
     while (total > G) {  // warp-uniform
@@ -227,6 +246,7 @@ __device__ __forceinline__ void pf_fill_chunk_table(const MixedParams& p, int* t
         tot[3] = longest;
         tot[4] = shortest;
         tot[5] = n_whole == 0 ? k0 : 1;
+        tot[6] = G;
     }
 }
 
@@ -242,7 +262,7 @@ __device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p, uint32_t ta
         plan.longest = lds_s32(tot + 12);
         plan.shortest = lds_s32(tot + 16);
         plan.pieces = lds_s32(tot + 20);
-        plan.ctas = (int)gridDim.x;
+        plan.ctas = lds_s32(tot + 24);
         return plan;
     }
     int G = (int)gridDim.x;
@@ -254,21 +274,11 @@ __device__ __forceinline__ PfPlan pf_make_plan(const MixedParams& p, uint32_t ta
         plan.longest = pf_steps_of_rank(p.group, p.cP[0], p.cC[0], n_tp, 0);
         plan.shortest = pf_steps_of_rank(p.group, p.cP[0], p.cC[0], n_tp, n_tp - 1);
     }
-    bool rounds = false;
-    float decode_steps = 0.f;  // the decode phase at the full streaming rate, in steps of an entry
-    if (p.n > 0) decode_steps = (float)__ldg(p.decode_page_indptr + p.n) * (float)p.Hkv * p.steps_per_stage;
-    if (p.n > 0 && plan.n_items >= G) {  // at least one whole round of items beside decode requests
-        // work in CTA-steps: the items (their lengths fall linearly with the rank) and the decode pages, at the rate of
-        // one CTA and with every CTA drawing 1 / G of the full rate
-        const float wp = 0.5f * (float)(plan.longest + plan.shortest) * (float)plan.n_items;
-        const float wd = decode_steps * (float)kDecodeCtasAtFullRate, wd_all = decode_steps * (float)G;
-        // CTA time the launch saves when few CTAs stream.  Entries run slower while pages are streamed beside them, so
-        // below a fifth of the launch the plain order (every CTA turns to the decode units after its entries) is kept;
-        // it is also kept beside a decode phase so short that latency, not the streaming rate, bounds it.
-        rounds = decode_steps >= kDecodeCtasMinSteps && wd_all - wd >= kDecodeCtasMinGain * (wp + wd_all);
-        // d CTAs streaming for the whole launch finish with the others when d / G is the decode share of the work
-        if (rounds) G -= min(min(kDecodeCtasAtFullRate, G / 2), (int)(wd * (float)G / (wp + wd) + 0.5f));
-    }
+    const float decode_steps = pf_decode_steps(p);
+    const int entry_ctas = pf_entry_ctas(p, G, plan.n_items, 0.5f * (float)(plan.longest + plan.shortest) * (float)plan.n_items,
+                                         decode_steps);
+    const bool rounds = entry_ctas < G;  // whole rounds of items (their lengths fall linearly with the rank) beside decode CTAs
+    G = entry_ctas;
     plan.ctas = G;
     const int r = plan.n_items % G;
     plan.n_whole = plan.n_items - r;

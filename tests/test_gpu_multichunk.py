@@ -56,6 +56,10 @@ CASES = {
     "long_end_new_start": (W.AttnShape(8, 2, 128), 400, [17, 300], [(3400, 70), (0, 50)]),
     "three_piece_counts": (W.AttnShape(8, 2, 128), 900, [64], [(8000, 100), (3300, 64), (0, 30)]),
     "pieces_trimmed_to_grid": (W.AttnShape(16, 16, 64), 1000, [100], [(9000, 300), (4000, 500)]),
+    # more work items (176) than SMs beside 780 MB of decode pages: some CTAs take no chunk-prefill entry and stream
+    # decode pages from the start, the whole rounds and the leftover pieces are shared by the others
+    "entry_ctas_beside_decode_pages": (W.AttnShape(16, 8, 128), 12400, [16000 - 111 * i for i in range(12)],
+                                       [(1000, 900), (0, 800), (300, 800)]),
 }
 
 
