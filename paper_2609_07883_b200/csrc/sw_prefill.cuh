@@ -92,20 +92,21 @@ __device__ __forceinline__ bool pf_wait(const PfShared& sh, int bar, uint32_t pa
 
 // ---- work decomposition -------------------------------------------------------------------------------------------
 // Items (one KV head x 256 query rows) are ordered longest first: rank 0 is the last 256-row group of the chunk.
-// A "step" is one 128-key KV tile of one item.  CTAs pull entries from a global counter.  The first n_whole
-// entries are whole items; the remaining r = n_items mod gridDim items (all of them when there are fewer items than
-// CTAs) would leave most SMs idle in the last wave, so each of them is cut along the KV axis into k pieces that run
-// side by side; every piece publishes a partial (m, l, O) and the last piece of an item to arrive merges them.
-// CTAs working at the same time thus stay at similar KV positions (their K/V tiles meet in L2).
+// A "step" is one 128-key KV tile of one item.  The G CTAs that take entries (PfPlan::ctas) pull them from a global
+// counter.  The first n_whole entries are whole items; the remaining r = n_items mod G items (all of them when there
+// are fewer items than CTAs) would leave most SMs idle in the last wave, so each of them is cut along the KV axis into k
+// pieces that run side by side; every piece publishes a partial (m, l, O) and the last piece of an item to arrive
+// merges them.  CTAs working at the same time thus stay at similar KV positions (their K/V tiles meet in L2).
 constexpr int kPfMinPieceSteps = 4;   // never pieces shorter than this many KV steps
 constexpr int kPfPieceCost = 1;       // steps' worth of work that cutting an item into one more piece costs
 // Whole rounds of items beside decode requests: the decode pages need the memory system, not the SMs, and about
 // kDecodeCtasAtFullRate CTAs' rings of page copies already draw the full rate.  So a few CTAs take no chunk-prefill work
-// at all and stream decode pages from the start, as many as it takes for the two kinds of work to end together; the
-// leftover items of the others' last round are cut into pieces that may run in several rounds.
+// at all and stream decode pages from the start, as many as it takes for the two kinds of work to end together (G is
+// the grid less those CTAs); the leftover items of the others' last round are cut into pieces that may run in several
+// rounds.  Whoever runs out of its own kind of work takes the other.
 constexpr int kDecodeCtasAtFullRate = 64;
-constexpr float kDecodeCtasMinGain = 0.20f;
-constexpr float kDecodeCtasMinSteps = 48.f;
+constexpr float kDecodeCtasMinGain = 0.20f;   // share of the launch's CTA time the rule must save to be applied
+constexpr float kDecodeCtasMinSteps = 48.f;   // and the shortest decode phase (at the full rate, in steps of an entry)
 constexpr int kPfMinRoundPieceSteps = 24;  // pieces that run in several rounds: at least this many KV steps each
 constexpr int kPfMaxRoundPieces = 12;
 
