@@ -52,9 +52,11 @@ WsLayout ws_layout(const sw_layout& l, int max_chunk, int max_decode, int64_t ma
     // 256-row groups of the chunks of one iteration: every chunk may end in a ragged group
     const size_t groups = ((size_t)max_chunk + (256 / g) - 1) / (256 / g) + sw::kMaxChunks;
     w.pf_tickets = off; off = align_up(off + std::max<size_t>(1, groups) * l.num_kv_heads * 2 * 4, 256);
-    // pieces of items publish partial results: one slot per CTA, more where a chunk can hold a whole round of items
-    // (its leftover items may then be cut into pieces that run in several rounds)
-    w.pf_slots = groups * l.num_kv_heads >= 64 ? sw::kPfRoundSlots : sw::kMaxCtas;
+    // pieces of items publish partial results: one slot per CTA, more where a single chunk can hold a whole round of
+    // items (its leftover items may then be cut into pieces that run in several rounds; the plan never uses more slots
+    // than it is given)
+    const size_t single_chunk_items = ((size_t)max_chunk + (256 / g) - 1) / (256 / g) * l.num_kv_heads;
+    w.pf_slots = single_chunk_items >= 96 ? sw::kPfRoundSlots : sw::kMaxCtas;
     w.pf_ml = off;    off = align_up(off + (size_t)w.pf_slots * 2 * 256 * 4, 256);
     w.pf_o = off;     off = align_up(off + (max_chunk > 0 ? (size_t)w.pf_slots * 2 * 128 * l.head_dim * 4 : 0), 256);
     w.st_q = off;     off = align_up(off + rows * l.num_q_heads * l.head_dim * 2, 256);
