@@ -133,6 +133,10 @@ cudaError_t launch_kv_append(const AppendParams& p, int num_sms, cudaStream_t st
 // against a plain copy on B200: 6.2 of 8.2 TB/s), and a 128-key step of a chunk-prefill entry takes about 4300 SM
 // cycles while other CTAs stream decode pages (measured; 2.2 us at 1965 MHz).
 inline void device_timing(int mem_clock_khz, int bus_width_bits, int sm_clock_khz, int head_dim, float* stage_us, float* step_us) {
+    // a driver that reports no clock leaves the plan with B200's nominal figures rather than with a division by zero
+    if (mem_clock_khz <= 0) mem_clock_khz = 3996000;
+    if (bus_width_bits <= 0) bus_width_bits = 8192;
+    if (sm_clock_khz <= 0) sm_clock_khz = 1965000;
     const double bytes_per_us = 0.76 * 2.0 * (double)mem_clock_khz * 1e3 * ((double)bus_width_bits / 8.0) / 1e6;
     const double stage_bytes = 2.0 * kPageSize * head_dim * 2;   // K and V rows of one head in a page
     *stage_us = (float)(stage_bytes / bytes_per_us);
