@@ -368,7 +368,8 @@ __device__ __forceinline__ void issue_page(const CUtensorMap* kvp_map, const War
         const uint32_t stage = issue_it % kStages;
         const uint32_t bar = ring.bar + stage * 8;
         mbar_arrive_expect_tx(bar, Geo<D>::kStageBytes);
-        tma_load_5d(ring.buf + stage * Geo<D>::kStageBytes, kvp_map, bar, 0, 0, 0, 2 * page, kvh);
+        // a decode page is read once: evict-first keeps it from pushing the chunk's K/V tiles out of L2
+        tma_load_5d_hint(ring.buf + stage * Geo<D>::kStageBytes, kvp_map, bar, 0, 0, 0, 2 * page, kvh, l2_policy_evict_first());
     }
 }
 
