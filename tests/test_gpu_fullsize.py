@@ -119,6 +119,55 @@ def test_whole_rounds_of_items_beside_many_decode_pages(gpu, oracle, C, P, n, L,
     run_case(gpu, oracle, batch, pairs, 150 + n, f"C={C} P={P} beside {n} decodes of up to {L} tokens", fused=fused)
 
 
+@pytest.mark.parametrize("case", ["pieces_in_rounds", "chat", "one_long_request"])
+def test_launches_stay_inside_the_workspace(gpu, oracle, case):
+    """The context is created on the middle of a larger buffer whose first and last MiB hold a pattern: after an iteration
+    that uses the scratch areas to the full (186 partial results of chunk-prefill pieces; the chat iteration; one request
+    cut into about 150 units per KV head) the pattern is untouched and the results match the oracle."""
+    import ctypes as C
+
+    import torch
+
+    from paper_2609_07883_b200 import binding as B
+
+    class GuardedContext(B.Context):
+        GUARD = 1 << 20
+
+        def __init__(self, shape, num_pages, max_chunk, max_decode, max_pages):
+            self.shape = shape
+            self.layout = B.make_layout(shape, num_pages)
+            self.device = torch.device("cuda", 0)
+            self.nbytes = B.sw_workspace_bytes(self.layout, max_chunk, max_decode, max_pages)
+            assert self.nbytes > 0
+            self.whole = torch.full((self.nbytes + 2 * self.GUARD,), 0xA5, dtype=torch.uint8, device=self.device)
+            self.workspace = self.whole[self.GUARD:self.GUARD + self.nbytes]
+            handle = C.c_void_p()
+            st = B._lib.sw_create(C.byref(self.layout), 0, self.workspace.data_ptr(), self.nbytes, max_chunk, max_decode,
+                                  max_pages, C.byref(handle))
+            assert st == B.SW_OK, B.sw_last_error()
+            self.handle = handle
+
+        def guards_intact(self):
+            g, n = self.GUARD, self.nbytes
+            return bool((self.whole[:g] == 0xA5).all().item()) and bool((self.whole[g + n:] == 0xA5).all().item())
+
+    rng = np.random.default_rng(21)
+    if case == "pieces_in_rounds":
+        C_, P, n, L = 2048, 12288, 35, 20000
+        lens = [L - (i * 37) % (L // 4) for i in range(n)]
+        batch = W.make_batch(W.LLAMA, sum(-(-x // 16) for x in lens) + (P + C_) // 16 + 64, lens, P, C_, rng)
+    elif case == "chat":
+        batch = W.chat_batch(n=64, chunk_len=512, prefix_len=512, rng=rng)
+    else:
+        batch = W.make_batch(W.LLAMA, 20000 // 16 + 72, [20000], 0, 0, rng)
+    total_pages = int(batch.prefill_pages.shape[0] + batch.decode_pages.shape[0])
+    ctx = GuardedContext(batch.shape, batch.num_pages, max(batch.chunk_len, 1), max(batch.num_decode, 1), total_pages + 16)
+    pairs = sample_pairs(batch, np.random.default_rng(22), gpu.boundary_rows(batch.chunk_len, batch.shape.group)[::4], 8)
+    for fused in (False, True):
+        run_case(gpu, oracle, batch, pairs, 170, f"guarded workspace, {case}, fused={fused}", fused=fused, ctx=ctx)
+        assert ctx.guards_intact(), f"{case}: a launch wrote outside the workspace"
+
+
 def test_page_ids_above_two_to_the_twenty(gpu, oracle):
     """A 70 GB pool (1.1 M pages of 64 KB) with the live pages scattered over all of it: byte offsets pass 2^36."""
     import torch
