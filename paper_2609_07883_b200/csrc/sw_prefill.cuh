@@ -107,6 +107,8 @@ constexpr int kPfPieceCost = 1;       // steps' worth of work that cutting an it
 constexpr int kDecodeCtasAtFullRate = 64;
 constexpr float kDecodeCtasMinGain = 0.20f;   // share of the launch's CTA time the rule must save to be applied
 constexpr float kDecodeCtasMinSteps = 48.f;   // and the shortest decode phase (at the full rate, in steps of an entry)
+constexpr float kEntryCostSteps = 3.f;        // fill and drain of an entry, in steps
+constexpr float kEntrySafety = 1.25f;
 constexpr int kPfMinRoundPieceSteps = 24;  // pieces that run in several rounds: at least this many KV steps each
 constexpr int kPfMaxRoundPieces = 12;
 
@@ -171,7 +173,14 @@ __device__ __forceinline__ int pf_entry_ctas(const MixedParams& p, int G, int n_
     // it is also kept beside a decode phase so short that latency, not the streaming rate, bounds it.
     if (decode_steps < kDecodeCtasMinSteps || wd_all - wd < kDecodeCtasMinGain * (wp + wd_all)) return G;
     // d CTAs streaming for the whole launch finish with the others when d / G is the decode share of the work
-    return G - min(min(kDecodeCtasAtFullRate, G / 2), (int)(wd * (float)G / (wp + wd) + 0.5f));
+    const int d = (int)(wd * (float)G / (wp + wd) + 0.5f);
+    if (d < kDecodeCtasAtFullRate) return G - min(d, G / 2);
+    // The decode pages are the longer part: kDecodeCtasAtFullRate streaming CTAs or more draw the full rate, so the launch
+    // cannot end before decode_steps, and the entries only have to be done by then.  They get as many CTAs as that takes
+    // (every entry counted with its fill and drain, and with a margin: entries run slower beside streaming CTAs), at
+    // least an eighth of the grid and at most what the full rate leaves.
+    const int need = (int)ceilf(kEntrySafety * (wp + kEntryCostSteps * (float)n_items) / decode_steps);
+    return min(max(need, max(1, G / 8)), G - min(kDecodeCtasAtFullRate, G / 2));
 }
 __device__ __forceinline__ float pf_decode_steps(const MixedParams& p) {  // the decode phase at the full rate, in steps
     return p.n > 0 ? (float)__ldg(p.decode_page_indptr + p.n) * (float)p.Hkv * p.steps_per_stage : 0.f;

@@ -103,7 +103,8 @@ def test_long_context_workload_large_chunks(gpu, oracle):
     (2048, 8192, 96, 4000, False),      # leftover items cut in two, side by side
     (2048, 12288, 35, 20000, True),     # about 60 leftover items cut in three: 180 pieces for the 98 CTAs that take them
     (2048, 16384, 47, 20000, False),    # about 60 leftover items cut in three to five, for 97 CTAs
-], ids=["whole_items", "two_pieces", "pieces_in_rounds", "more_pieces_in_rounds"])
+    (2048, 0, 128, 3200, True),         # the decode pages are the longer part: the 256 short items run on about 30 CTAs
+], ids=["whole_items", "two_pieces", "pieces_in_rounds", "more_pieces_in_rounds", "entries_on_few_ctas"])
 def test_whole_rounds_of_items_beside_many_decode_pages(gpu, oracle, C, P, n, L, fused):
     """A chunk of at least one whole round of work items (one per SM) beside decode requests whose pages are a tenth of
     the launch or more: some CTAs take no chunk-prefill entry and stream decode pages from the start, the others share
